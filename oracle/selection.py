@@ -79,11 +79,15 @@ def stage1_keys(mask: np.ndarray, conf: np.ndarray, sigma: float) -> np.ndarray:
     return key
 
 
+SCORE_CAP = np.float32(262144.0)   # 2^18: keeps the fixed-point mass of 8192 positions inside 64 bits
+
+
 def _clean_score(x: np.ndarray) -> np.ndarray:
-    """Scores that are NaN or negative count as 0 (they cannot be ordered as masses)."""
+    """Scores that are NaN, negative or infinite count as 0 (they cannot be ordered as masses);
+    finite ones are capped at 2^18 (a rollout score never exceeds the sequence length)."""
     x = np.asarray(x, dtype=np.float32).copy()
-    x[~(x > 0)] = 0.0
-    return x
+    x[~((x > 0) & np.isfinite(x))] = 0.0
+    return np.minimum(x, SCORE_CAP)
 
 
 def stage1_select(mask: np.ndarray, conf: np.ndarray, k: int, sigma: float,

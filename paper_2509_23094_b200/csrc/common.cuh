@@ -1,0 +1,101 @@
+// Shared declarations of the d2c CUDA sources: error plumbing, small device helpers and the
+// launchers each .cu file exposes to the C-ABI layer (d2c_api.cu).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "../../include/d2c.h"
+
+typedef __nv_bfloat16 bf16;
+
+namespace d2c {
+
+// Text of the last error raised outside any context (thread local).
+void set_global_error(const char* fmt, ...);
+const char* global_error();
+
+#define D2C_CUDA_OK(expr)                                                              \
+  do {                                                                                 \
+    cudaError_t e__ = (expr);                                                          \
+    if (e__ != cudaSuccess) {                                                          \
+      d2c::set_global_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__),   \
+                            __FILE__, __LINE__);                                       \
+      return D2C_ECUDA;                                                                \
+    }                                                                                  \
+  } while (0)
+
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- selection (select.cu) -------------------------------------------------------------------
+struct SelectArgs {
+  const uint8_t* mask; const float* conf; const float* c; const float* override_key;
+  const int32_t* forced; const int32_t* forced_off;
+  int batch, seq_len, k; float p; int stage2_candidates;
+  const uint32_t* phi_q30; int phi_len;          // phi table in 2^-30 fixed point, entries [0, phi_len)
+  float* key; int32_t* sel_idx; int32_t* row_seq; int32_t* row_off; int32_t* lm_rows; int32_t* lm_off;
+  int32_t* slot_of_pos;
+  int32_t* rank_s; int32_t* rank_lm; int32_t* n_b; int32_t* nm_b;   // scratch [B][L],[B][L],[B],[B]
+};
+int launch_select(const SelectArgs& a, cudaStream_t st);
+// Fills tab[0..len) with floor(exp(-r^2/(2 sigma^2)) * 2^30 + 0.5); returns the first r whose entry is 0 (or len).
+int build_phi_table(float sigma, uint32_t* tab, int len);
+
+// ---- row kernels (rows.cu) -------------------------------------------------------------------
+int launch_gather_norm(const bf16* h0, const int32_t* sel_idx, const int32_t* row_seq, const int32_t* n_rows,
+                       int max_rows, int seq_len, int d, const bf16* gain, float eps, bf16* x, bf16* xn,
+                       cudaStream_t st);
+int launch_rmsnorm(const bf16* x, const int32_t* row_map, const int32_t* n_rows, int max_rows, int d,
+                   const bf16* gain, float eps, bf16* xn, cudaStream_t st);
+int launch_rope_table(float2* tab, int max_seq, int head_dim, float base, cudaStream_t st);
+int launch_rope_scatter(bf16* qkv, const int32_t* sel_idx, const int32_t* row_seq, const int32_t* n_rows,
+                        int max_rows, int hq, int hkv, int dh, const float2* rope, bf16* kc, bf16* vc,
+                        int cache_seq, cudaStream_t st);
+
+// ---- GEMMs (gemm_mma.cu, gemm_tc.cu) -----------------------------------------------------------
+enum GemmEpilogue { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_LMSTATS = 3 };
+struct GemmArgs {
+  const bf16* A; int lda;            // [max_rows][K]
+  const bf16* W; const bf16* W2;     // [N][K]; W2 = the "up" matrix for EPI_SWIGLU
+  const bf16* bias;                  // [N] or null (EPI_STORE)
+  bf16* C; int ldc;                  // output (EPI_STORE / EPI_RESIDUAL: C += ; EPI_SWIGLU: silu(AW^T)*(AW2^T))
+  const int32_t* n_rows; int max_rows; int N; int K;
+  // EPI_LMSTATS: per (row, 128-column tile) running max / sum of exp / arg-max, optional raw logits
+  float* st_max; float* st_sum; int32_t* st_arg; float* logits; int n_tiles;
+};
+int launch_gemm_mma(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st);
+
+// ---- attention (attention.cu) ----------------------------------------------------------------
+struct AttnArgs {
+  const bf16* q; int ldq; const bf16* kc; const bf16* vc; const int32_t* row_off;
+  int batch, seq_len, cache_seq, hq, hkv, dh; int max_rows_per_seq;
+  bf16* o; float* lse; float* abar;      // abar may be null (layers outside the rollout)
+};
+int launch_attention(const AttnArgs& a, cudaStream_t st);
+
+// ---- LM head statistics (lmhead.cu) ------------------------------------------------------------
+int launch_lm_reduce(const float* st_max, const float* st_sum, const int32_t* st_arg, int n_tiles,
+                     const int32_t* n_rows, int max_rows, const int32_t* lm_rows, const int32_t* sel_idx,
+                     const int32_t* row_seq, int seq_len, float* conf, int32_t* pred, cudaStream_t st);
+
+// ---- rollout (rollout.cu) ----------------------------------------------------------------------
+struct RolloutArgs {
+  const float* abar; size_t layer_stride; int n_layers; const int32_t* sel_idx; const int32_t* row_off;
+  int batch, seq_len; float* c; float* u0; float* u1; float* partial; int n_split;
+};
+int launch_rollout(const RolloutArgs& a, cudaStream_t st);
+static const int kRolloutSplit = 16;
+
+}  // namespace d2c
+
+namespace d2c {
+// ---- commit helper (commit.cu) -------------------------------------------------------------------
+int launch_commit(int batch, int seq_len, int d, int rule, float threshold, const int32_t* slot_of_pos,
+                  const float* conf, const int32_t* pred, const uint32_t* phi, int phi_len, const bf16* embed,
+                  bf16* h0, uint8_t* mask, int32_t* tokens, int32_t* committed, cudaStream_t st);
+// ---- tcgen05 GEMM (gemm_tc.cu) -------------------------------------------------------------------
+int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st);
+}  // namespace d2c

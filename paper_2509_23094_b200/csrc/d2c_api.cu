@@ -1,0 +1,346 @@
+// C-ABI layer of the d2Cache step: argument validation, the carve-up of the caller's workspace and
+// the launch sequence of one step.  No device memory is allocated here.
+#include <math.h>
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace d2c {
+
+static thread_local char g_err[512] = "";
+void set_global_error(const char* fmt, ...) {
+  va_list ap; va_start(ap, fmt); vsnprintf(g_err, sizeof(g_err), fmt, ap); va_end(ap);
+}
+const char* global_error() { return g_err; }
+
+// Hands out 256-byte aligned pieces of a buffer; with base == null it only measures.
+struct Carver {
+  char* base; size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+  template <typename T> T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+struct Buffers {
+  bf16 *kcache, *vcache; float *conf, *c, *key; int32_t *pred, *status;
+  int32_t *sel_idx, *row_seq, *row_off, *lm_rows, *lm_off, *slot_of_pos, *rank_s, *rank_lm, *n_b, *nm_b;
+  uint32_t* phi; float2* rope;
+  bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar;
+  float *st_max, *st_sum; int32_t* st_arg;
+  float *u0, *u1, *partial;
+  bf16* h0_stage; uint8_t* mask_stage; int32_t *forced_stage, *forced_off_stage; float *okey_stage, *oc_stage;
+  int32_t* committed_stage;
+};
+
+static int rollout_depth(const d2c_config& c) {
+  return (c.rollout_layers > 0 && c.rollout_layers < c.n_layers) ? c.rollout_layers : c.n_layers;
+}
+static int lm_tiles(int vocab) { return ceil_div(vocab, 128); }
+
+static size_t carve(const d2c_config& c, void* base, Buffers* out) {
+  Carver w(base);
+  Buffers b;
+  const size_t B = c.max_batch, L = c.max_seq, R = B * L, d = c.d_model;
+  const size_t kv = (size_t)c.n_kv_heads * c.head_dim, qkv_out = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  b.kcache = w.take<bf16>((size_t)c.n_layers * R * kv);
+  b.vcache = w.take<bf16>((size_t)c.n_layers * R * kv);
+  b.conf = w.take<float>(R); b.c = w.take<float>(R); b.key = w.take<float>(R);
+  b.pred = w.take<int32_t>(R); b.status = w.take<int32_t>(4);
+  b.sel_idx = w.take<int32_t>(R); b.row_seq = w.take<int32_t>(R); b.row_off = w.take<int32_t>(B + 1);
+  b.lm_rows = w.take<int32_t>(R); b.lm_off = w.take<int32_t>(B + 1); b.slot_of_pos = w.take<int32_t>(R);
+  b.rank_s = w.take<int32_t>(R); b.rank_lm = w.take<int32_t>(R); b.n_b = w.take<int32_t>(B); b.nm_b = w.take<int32_t>(B);
+  b.phi = w.take<uint32_t>(L); b.rope = w.take<float2>(L * (c.head_dim / 2));
+  b.x = w.take<bf16>(R * d); b.xn = w.take<bf16>(R * d); b.qkv = w.take<bf16>(R * qkv_out);
+  b.o = w.take<bf16>(R * (size_t)c.n_q_heads * c.head_dim); b.hmid = w.take<bf16>(R * (size_t)c.d_ffn);
+  b.xm = w.take<bf16>(R * d); b.lse = w.take<float>(R * (size_t)c.n_q_heads);
+  b.abar = w.take<float>((size_t)rollout_depth(c) * R * L);
+  const size_t nt = lm_tiles(c.vocab);
+  b.st_max = w.take<float>(R * nt); b.st_sum = w.take<float>(R * nt); b.st_arg = w.take<int32_t>(R * nt);
+  b.u0 = w.take<float>(R); b.u1 = w.take<float>(R);
+  b.partial = w.take<float>((size_t)kRolloutSplit * R + (R + 3) / 4);     // partial sums + selected-flag bytes
+  b.h0_stage = w.take<bf16>(R * d); b.mask_stage = w.take<uint8_t>(R);
+  b.forced_stage = w.take<int32_t>(R); b.forced_off_stage = w.take<int32_t>(B + 1);
+  b.okey_stage = w.take<float>(R); b.oc_stage = w.take<float>(R); b.committed_stage = w.take<int32_t>(B);
+  if (out) *out = b;
+  return align_up(w.off, 256);
+}
+
+static const char* check_config(const d2c_config* c) {
+  if (!c) return "config is null";
+  if (c->n_layers < 1 || c->d_model < 64 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 64 || c->vocab < 2)
+    return "non-positive model dimension";
+  if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
+  if (c->d_model % 64 || c->d_ffn % 64 || (c->n_q_heads * c->head_dim) % 64) return "d_model, d_ffn and n_q_heads*head_dim must be multiples of 64";
+  if (c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c->vocab & 1) return "vocab must be even";
+  if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
+  if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
+  if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
+  if (c->rollout_layers < 0 || c->flags != 0) return "rollout_layers >= 0 and flags == 0 required";
+  return nullptr;
+}
+
+}  // namespace d2c
+
+using namespace d2c;
+
+struct d2c_ctx {
+  d2c_config cfg;
+  std::vector<const bf16*> wqkv, bqkv, wo, w_gate, w_up, w_down, g_attn, g_ffn;
+  const bf16 *g_final, *w_lm;
+  cudaStream_t stream;
+  Buffers buf;
+  int phi_len;
+  char err[512];
+};
+
+static int fail(d2c_ctx* ctx, int code, const char* fmt, ...) {
+  char tmp[512];
+  va_list ap; va_start(ap, fmt); vsnprintf(tmp, sizeof(tmp), fmt, ap); va_end(ap);
+  if (ctx) { strncpy(ctx->err, tmp, sizeof(ctx->err) - 1); ctx->err[sizeof(ctx->err) - 1] = 0; }
+  set_global_error("%s", tmp);
+  return code;
+}
+// Propagates an error raised by a launcher (its text is in the thread-local slot).
+static int pass(d2c_ctx* ctx, int rc) {
+  if (rc != D2C_OK && ctx) { strncpy(ctx->err, global_error(), sizeof(ctx->err) - 1); ctx->err[sizeof(ctx->err) - 1] = 0; }
+  return rc;
+}
+#define D2C_TRY(ctx, expr) do { int rc__ = (expr); if (rc__ != D2C_OK) return pass((ctx), rc__); } while (0)
+
+extern "C" {
+
+size_t d2c_workspace_bytes(const d2c_config* cfg) {
+  if (check_config(cfg)) return 0;
+  return carve(*cfg, nullptr, nullptr);
+}
+
+int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, size_t workspace_bytes,
+               void* cuda_stream, d2c_ctx** out) {
+  if (!out) return fail(nullptr, D2C_EINVAL, "d2c_create: out is null");
+  *out = nullptr;
+  if (const char* why = check_config(cfg)) return fail(nullptr, cfg ? D2C_ESHAPE : D2C_EINVAL, "d2c_create: %s", why);
+  if (!w || !workspace) return fail(nullptr, D2C_EINVAL, "d2c_create: weights or workspace is null");
+  if (reinterpret_cast<uintptr_t>(workspace) % 256) return fail(nullptr, D2C_EINVAL, "d2c_create: workspace must be 256-byte aligned");
+  const size_t need = carve(*cfg, nullptr, nullptr);
+  if (workspace_bytes < need) return fail(nullptr, D2C_ECAPACITY, "d2c_create: workspace %zu bytes < %zu needed", workspace_bytes, need);
+  if (!w->wqkv || !w->wo || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn || !w->g_ffn || !w->g_final || !w->w_lm ||
+      (cfg->qkv_bias && !w->bqkv))
+    return fail(nullptr, D2C_EINVAL, "d2c_create: a weight pointer is null");
+  d2c_ctx* ctx = new (std::nothrow) d2c_ctx();
+  if (!ctx) return fail(nullptr, D2C_EINVAL, "d2c_create: out of host memory");
+  ctx->cfg = *cfg; ctx->err[0] = 0;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const void* ptrs[] = {w->wqkv[l], w->wo[l], w->w_gate[l], w->w_up[l], w->w_down[l], w->g_attn[l], w->g_ffn[l]};
+    for (const void* p : ptrs)
+      if (!p || reinterpret_cast<uintptr_t>(p) % 16) { delete ctx; return fail(nullptr, D2C_EINVAL, "d2c_create: layer %d weight pointer null or not 16-byte aligned", l); }
+    ctx->wqkv.push_back((const bf16*)w->wqkv[l]); ctx->wo.push_back((const bf16*)w->wo[l]);
+    ctx->w_gate.push_back((const bf16*)w->w_gate[l]); ctx->w_up.push_back((const bf16*)w->w_up[l]);
+    ctx->w_down.push_back((const bf16*)w->w_down[l]); ctx->g_attn.push_back((const bf16*)w->g_attn[l]);
+    ctx->g_ffn.push_back((const bf16*)w->g_ffn[l]);
+    ctx->bqkv.push_back(cfg->qkv_bias ? (const bf16*)w->bqkv[l] : nullptr);
+    if (cfg->qkv_bias && !w->bqkv[l]) { delete ctx; return fail(nullptr, D2C_EINVAL, "d2c_create: layer %d bias is null", l); }
+  }
+  ctx->g_final = (const bf16*)w->g_final; ctx->w_lm = (const bf16*)w->w_lm;
+  carve(*cfg, workspace, &ctx->buf);
+  cudaError_t e = cudaMemsetAsync(workspace, 0, need, ctx->stream);
+  if (e == cudaSuccess) {
+    std::vector<uint32_t> tab(cfg->max_seq);
+    ctx->phi_len = build_phi_table(cfg->sigma, tab.data(), cfg->max_seq);
+    e = cudaMemcpyAsync(ctx->buf.phi, tab.data(), tab.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream);
+    if (e == cudaSuccess) {
+      int rc = launch_rope_table(ctx->buf.rope, cfg->max_seq, cfg->head_dim, cfg->rope_base, ctx->stream);
+      if (rc != D2C_OK) { delete ctx; return rc; }
+      e = cudaStreamSynchronize(ctx->stream);      // the host table above must outlive the copy
+    }
+  }
+  if (e != cudaSuccess) { delete ctx; return fail(nullptr, D2C_ECUDA, "d2c_create: %s", cudaGetErrorString(e)); }
+  *out = ctx;
+  return D2C_OK;
+}
+
+int d2c_destroy(d2c_ctx* ctx) {
+  if (!ctx) return D2C_EINVAL;
+  delete ctx;
+  return D2C_OK;
+}
+
+const char* d2c_last_error(const d2c_ctx* ctx) { return ctx ? ctx->err : global_error(); }
+
+int d2c_state_ptrs(d2c_ctx* ctx, d2c_state* out) {
+  if (!ctx || !out) return D2C_EINVAL;
+  const Buffers& b = ctx->buf;
+  out->kcache = b.kcache; out->vcache = b.vcache; out->conf = b.conf; out->pred = b.pred; out->c = b.c; out->key = b.key;
+  out->sel_idx = b.sel_idx; out->row_off = b.row_off; out->lm_rows = b.lm_rows; out->lm_off = b.lm_off;
+  out->abar = b.abar; out->lse = b.lse; out->status = b.status;
+  return D2C_OK;
+}
+
+int d2c_sync_status(d2c_ctx* ctx) {
+  if (!ctx) return D2C_EINVAL;
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_sync_status: %s", cudaGetErrorString(e));
+  int32_t st[4];
+  e = cudaMemcpy(st, ctx->buf.status, sizeof(st), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_sync_status: %s", cudaGetErrorString(e));
+  if (st[0] != 0) return fail(ctx, st[0], "device status %d raised at site %d", st[0], st[1]);
+  return D2C_OK;
+}
+
+static int check_step_args(d2c_ctx* ctx, const d2c_step_args* a) {
+  if (!ctx) return D2C_EINVAL;
+  if (!a) return fail(ctx, D2C_EINVAL, "d2c_step: args is null");
+  if (a->batch < 1 || a->seq_len < 1) return fail(ctx, D2C_EINVAL, "d2c_step: batch %d / seq_len %d must be positive", a->batch, a->seq_len);
+  if (a->batch > ctx->cfg.max_batch || a->seq_len > ctx->cfg.max_seq)
+    return fail(ctx, D2C_ECAPACITY, "d2c_step: batch %d x seq_len %d exceeds the context's %d x %d", a->batch, a->seq_len, ctx->cfg.max_batch, ctx->cfg.max_seq);
+  if (!a->h0 || !a->mask) return fail(ctx, D2C_EINVAL, "d2c_step: h0 or mask is null");
+  if (a->k < 0) return fail(ctx, D2C_EINVAL, "d2c_step: k = %d is negative", a->k);
+  if (isnan(a->p)) return fail(ctx, D2C_EINVAL, "d2c_step: p is NaN");
+  if ((a->forced == nullptr) != (a->forced_off == nullptr)) return fail(ctx, D2C_EINVAL, "d2c_step: forced and forced_off must be given together");
+  return D2C_OK;
+}
+
+int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
+  D2C_TRY(ctx, check_step_args(ctx, a));
+  const d2c_config& c = ctx->cfg;
+  const Buffers& b = ctx->buf;
+  cudaStream_t st = ctx->stream;
+  const int B = a->batch, L = a->seq_len, R = B * L, d = c.d_model;
+  const int hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
+  const int qkv_out = (hq + 2 * hkv) * dh;
+  const size_t cache_layer = (size_t)c.max_batch * c.max_seq * hkv * dh;
+  bf16* x = (out && out->hidden_out) ? static_cast<bf16*>(out->hidden_out) : b.x;
+  if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(a->h0) % 16)
+    return fail(ctx, D2C_EINVAL, "d2c_step: h0 and hidden_out must be 16-byte aligned");
+
+  SelectArgs s{};
+  s.mask = a->mask; s.conf = b.conf; s.c = a->override_c ? a->override_c : b.c; s.override_key = a->override_key;
+  s.forced = a->forced; s.forced_off = a->forced_off; s.batch = B; s.seq_len = L; s.k = a->k; s.p = a->p;
+  s.stage2_candidates = c.stage2_candidates; s.phi_q30 = b.phi; s.phi_len = ctx->phi_len < L ? ctx->phi_len : L;
+  s.key = b.key; s.sel_idx = b.sel_idx; s.row_seq = b.row_seq; s.row_off = b.row_off; s.lm_rows = b.lm_rows;
+  s.lm_off = b.lm_off; s.slot_of_pos = b.slot_of_pos; s.rank_s = b.rank_s; s.rank_lm = b.rank_lm; s.n_b = b.n_b; s.nm_b = b.nm_b;
+  D2C_TRY(ctx, launch_select(s, st));
+  const int32_t* n_rows = b.row_off + B;
+  const int32_t* n_lm = b.lm_off + B;
+
+  D2C_TRY(ctx, launch_gather_norm((const bf16*)a->h0, b.sel_idx, b.row_seq, n_rows, R, L, d, ctx->g_attn[0], c.rms_eps, x, b.xn, st));
+  const int depth = rollout_depth(c);
+  for (int l = 0; l < c.n_layers; ++l) {
+    if (l > 0) D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
+    GemmArgs g{};
+    g.A = b.xn; g.lda = d; g.W = ctx->wqkv[l]; g.bias = ctx->bqkv[l]; g.C = b.qkv; g.ldc = qkv_out;
+    g.n_rows = n_rows; g.max_rows = R; g.N = qkv_out; g.K = d;
+    D2C_TRY(ctx, launch_gemm_mma(g, EPI_STORE, st));
+    bf16* kc = b.kcache + (size_t)l * cache_layer; bf16* vc = b.vcache + (size_t)l * cache_layer;
+    D2C_TRY(ctx, launch_rope_scatter(b.qkv, b.sel_idx, b.row_seq, n_rows, R, hq, hkv, dh, b.rope, kc, vc, c.max_seq, st));
+    AttnArgs at{};
+    at.q = b.qkv; at.ldq = qkv_out; at.kc = kc; at.vc = vc; at.row_off = b.row_off; at.batch = B; at.seq_len = L;
+    at.cache_seq = c.max_seq; at.hq = hq; at.hkv = hkv; at.dh = dh; at.max_rows_per_seq = L;
+    at.o = b.o; at.lse = b.lse; at.abar = l < depth ? b.abar + (size_t)l * c.max_batch * c.max_seq * c.max_seq : nullptr;
+    D2C_TRY(ctx, launch_attention(at, st));
+    GemmArgs go{};
+    go.A = b.o; go.lda = hq * dh; go.W = ctx->wo[l]; go.C = x; go.ldc = d; go.n_rows = n_rows; go.max_rows = R; go.N = d; go.K = hq * dh;
+    D2C_TRY(ctx, launch_gemm_mma(go, EPI_RESIDUAL, st));
+    D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_ffn[l], c.rms_eps, b.xn, st));
+    GemmArgs gf{};
+    gf.A = b.xn; gf.lda = d; gf.W = ctx->w_gate[l]; gf.W2 = ctx->w_up[l]; gf.C = b.hmid; gf.ldc = c.d_ffn;
+    gf.n_rows = n_rows; gf.max_rows = R; gf.N = c.d_ffn; gf.K = d;
+    D2C_TRY(ctx, launch_gemm_mma(gf, EPI_SWIGLU, st));
+    GemmArgs gd{};
+    gd.A = b.hmid; gd.lda = c.d_ffn; gd.W = ctx->w_down[l]; gd.C = x; gd.ldc = d; gd.n_rows = n_rows; gd.max_rows = R; gd.N = d; gd.K = c.d_ffn;
+    D2C_TRY(ctx, launch_gemm_mma(gd, EPI_RESIDUAL, st));
+  }
+  // Eq. 1 on the selected rows that are still masked
+  D2C_TRY(ctx, launch_rmsnorm(x, b.lm_rows, n_lm, R, d, ctx->g_final, c.rms_eps, b.xm, st));
+  GemmArgs gl{};
+  gl.A = b.xm; gl.lda = d; gl.W = ctx->w_lm; gl.n_rows = n_lm; gl.max_rows = R; gl.N = c.vocab; gl.K = d;
+  gl.st_max = b.st_max; gl.st_sum = b.st_sum; gl.st_arg = b.st_arg; gl.n_tiles = lm_tiles(c.vocab);
+  gl.logits = out ? out->logits : nullptr;
+  D2C_TRY(ctx, launch_gemm_mma(gl, EPI_LMSTATS, st));
+  D2C_TRY(ctx, launch_lm_reduce(b.st_max, b.st_sum, b.st_arg, gl.n_tiles, n_lm, R, b.lm_rows, b.sel_idx, b.row_seq, L, b.conf, b.pred, st));
+  // Eq. 6-9 for the next step's stage 2
+  RolloutArgs r{};
+  r.abar = b.abar; r.layer_stride = (size_t)c.max_batch * c.max_seq * c.max_seq; r.n_layers = depth; r.sel_idx = b.sel_idx;
+  r.row_off = b.row_off; r.batch = B; r.seq_len = L; r.c = b.c; r.u0 = b.u0; r.u1 = b.u1; r.partial = b.partial; r.n_split = kRolloutSplit;
+  D2C_TRY(ctx, launch_rollout(r, st));
+
+  if (out && out->sel_idx) {
+    cudaError_t e = cudaMemcpyAsync(out->sel_idx, b.sel_idx, (size_t)R * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
+  }
+  if (out && out->row_off) {
+    cudaError_t e = cudaMemcpyAsync(out->row_off, b.row_off, (size_t)(B + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
+  }
+  return D2C_OK;
+}
+
+int d2c_step_host(d2c_ctx* ctx, const d2c_step_args* h, const d2c_host_out* out) {
+  D2C_TRY(ctx, check_step_args(ctx, h));
+  const d2c_config& c = ctx->cfg;
+  const Buffers& b = ctx->buf;
+  cudaStream_t st = ctx->stream;
+  const size_t B = h->batch, L = h->seq_len, R = B * L;
+#define D2C_CP(dst, src, bytes, kind)                                                         \
+  do { cudaError_t e__ = cudaMemcpyAsync((dst), (src), (bytes), (kind), st);                  \
+       if (e__ != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e__)); } while (0)
+  d2c_step_args a = *h;
+  D2C_CP(b.h0_stage, h->h0, R * c.d_model * sizeof(bf16), cudaMemcpyHostToDevice); a.h0 = b.h0_stage;
+  D2C_CP(b.mask_stage, h->mask, R, cudaMemcpyHostToDevice); a.mask = b.mask_stage;
+  if (h->forced) {
+    int32_t n_forced = h->forced_off[B];
+    if (n_forced < 0 || (size_t)n_forced > R) return fail(ctx, D2C_EINVAL, "d2c_step_host: %d forced rows", n_forced);
+    D2C_CP(b.forced_off_stage, h->forced_off, (B + 1) * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (n_forced) D2C_CP(b.forced_stage, h->forced, (size_t)n_forced * sizeof(int32_t), cudaMemcpyHostToDevice);
+    a.forced = b.forced_stage; a.forced_off = b.forced_off_stage;
+  }
+  if (h->override_key) { D2C_CP(b.okey_stage, h->override_key, R * sizeof(float), cudaMemcpyHostToDevice); a.override_key = b.okey_stage; }
+  if (h->override_c) { D2C_CP(b.oc_stage, h->override_c, R * sizeof(float), cudaMemcpyHostToDevice); a.override_c = b.oc_stage; }
+  d2c_step_out dev_out{};
+  D2C_TRY(ctx, d2c_step(ctx, &a, &dev_out));
+  std::vector<int32_t> ro(B + 1);
+  D2C_CP(ro.data(), b.row_off, (B + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  cudaError_t e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e));
+  const size_t n = (size_t)ro[B];
+  if (out) {
+    if (out->row_off_host) memcpy(out->row_off_host, ro.data(), (B + 1) * sizeof(int32_t));
+    if (out->sel_idx_host && n) D2C_CP(out->sel_idx_host, b.sel_idx, n * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    if (out->hidden_out_host && n) D2C_CP(out->hidden_out_host, b.x, n * c.d_model * sizeof(bf16), cudaMemcpyDeviceToHost);
+    if (out->conf_host) {
+      for (size_t bb = 0; bb < B; ++bb) D2C_CP(out->conf_host + bb * L, b.conf + bb * L, L * sizeof(float), cudaMemcpyDeviceToHost);
+    }
+    if (out->pred_host) {
+      for (size_t bb = 0; bb < B; ++bb) D2C_CP(out->pred_host + bb * L, b.pred + bb * L, L * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    }
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e));
+  }
+#undef D2C_CP
+  return D2C_OK;
+}
+
+int d2c_commit(d2c_ctx* ctx, int32_t batch, int32_t seq_len, const void* embed_table, void* h0,
+               uint8_t* mask, int32_t* tokens, int32_t* committed, int32_t rule, float threshold) {
+  if (!ctx) return D2C_EINVAL;
+  if (!embed_table || !h0 || !mask || !tokens || !committed) return fail(ctx, D2C_EINVAL, "d2c_commit: null pointer");
+  if (batch < 1 || batch > ctx->cfg.max_batch || seq_len < 1 || seq_len > ctx->cfg.max_seq)
+    return fail(ctx, D2C_ECAPACITY, "d2c_commit: batch %d x seq_len %d out of range", batch, seq_len);
+  if (rule < 0 || rule > 2 || isnan(threshold)) return fail(ctx, D2C_EINVAL, "d2c_commit: rule %d / threshold", rule);
+  const Buffers& b = ctx->buf;
+  D2C_TRY(ctx, launch_commit(batch, seq_len, ctx->cfg.d_model, rule, threshold, b.slot_of_pos, b.conf, b.pred, b.phi,
+                             ctx->phi_len < seq_len ? ctx->phi_len : seq_len, (const bf16*)embed_table, (bf16*)h0, mask,
+                             tokens, committed, ctx->stream));
+  return D2C_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+// Eq. 1 from the per-tile statistics the LM-head GEMM leaves behind: for every row the running
+// maximum, its column and sum exp(x - max) of each 128-column tile are merged into the arg-max
+// token and its softmax probability 1 / sum_j exp(x_j - max).  The logits never reach HBM.
+#include "common.cuh"
+
+namespace d2c {
+
+// One warp per row.  lm_rows == null: results go to conf[r] / pred[r]; otherwise row lm_rows[r] of
+// the step is looked up and the result is scattered to its (sequence, position).
+__global__ void __launch_bounds__(128)
+lm_reduce_kernel(const float* __restrict__ st_max, const float* __restrict__ st_sum,
+                 const int32_t* __restrict__ st_arg, int n_tiles, const int32_t* __restrict__ n_rows,
+                 const int32_t* __restrict__ lm_rows, const int32_t* __restrict__ sel_idx,
+                 const int32_t* __restrict__ row_seq, int seq_len, float* __restrict__ conf,
+                 int32_t* __restrict__ pred) {
+  const int n = *n_rows, lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  for (int r = blockIdx.x * wpb + (threadIdx.x >> 5); r < n; r += gridDim.x * wpb) {
+    const size_t base = (size_t)r * n_tiles;
+    float mx = -INFINITY; int arg = 0x7fffffff;
+    for (int t = lane; t < n_tiles; t += 32) {
+      const float v = st_max[base + t]; const int a2 = st_arg[base + t];
+      if (v > mx || (v == mx && a2 < arg)) { mx = v; arg = a2; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float omx = __shfl_xor_sync(0xffffffffu, mx, o);
+      const int oarg = __shfl_xor_sync(0xffffffffu, arg, o);
+      if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+    }
+    float sum = 0.f;
+    for (int t = lane; t < n_tiles; t += 32) sum += st_sum[base + t] * __expf(st_max[base + t] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) {
+      size_t dst = (size_t)r;
+      if (lm_rows) { const int row = lm_rows[r]; dst = (size_t)row_seq[row] * seq_len + sel_idx[row]; }
+      conf[dst] = 1.f / sum;
+      pred[dst] = arg;
+    }
+  }
+}
+
+int launch_lm_reduce(const float* st_max, const float* st_sum, const int32_t* st_arg, int n_tiles,
+                     const int32_t* n_rows, int max_rows, const int32_t* lm_rows, const int32_t* sel_idx,
+                     const int32_t* row_seq, int seq_len, float* conf, int32_t* pred, cudaStream_t st) {
+  if (max_rows <= 0) return D2C_OK;
+  const int grid = ceil_div(max_rows, 4) < 148 * 4 ? ceil_div(max_rows, 4) : 148 * 4;
+  lm_reduce_kernel<<<grid, 128, 0, st>>>(st_max, st_sum, st_arg, n_tiles, n_rows, lm_rows, sel_idx, row_seq,
+                                         seq_len, conf, pred);
+  D2C_CUDA_OK(cudaGetLastError());
+  return D2C_OK;
+}
+
+}  // namespace d2c

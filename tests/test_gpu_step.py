@@ -1,0 +1,163 @@
+"""d2c_step against the oracle, end to end: prefill (all rows), partial steps, the degenerate steps."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_23094_b200 import inputs
+from gpu_util import ROW_TOL, Pair, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_state(pair, res, sel, mask=None):
+    """Cache rows of the selected positions, confidences, predictions and rollout scores."""
+    wl, shape = pair.wl, pair.shape
+    B, L = wl.batch, wl.seq_len
+    mask = pair.mask if mask is None else mask
+    kc = pair.ctx.view("kcache").float().cpu().numpy(); vc = pair.ctx.view("vcache").float().cpu().numpy()
+    conf = pair.ctx.view("conf", B, L).cpu().numpy(); pred = pair.ctx.view("pred", B, L).cpu().numpy()
+    c = pair.ctx.view("c", B, L).cpu().numpy()
+    kv = shape.n_kv_heads * shape.head_dim
+    for b in range(B):
+        S = sel[b]
+        for l in range(shape.n_layers):
+            assert row_rel_err(kc[l, b, S].reshape(len(S), kv), pair.ost.Kc[l, b, S].reshape(len(S), kv)) <= ROW_TOL, (l, b)
+            assert row_rel_err(vc[l, b, S].reshape(len(S), kv), pair.ost.Vc[l, b, S].reshape(len(S), kv)) <= ROW_TOL, (l, b)
+        lm = res.lm_rows[b]
+        if len(lm):
+            np.testing.assert_allclose(conf[b, lm], pair.ost.conf[b, lm], rtol=0.1, atol=1e-7)
+            # the predicted token must be (one of) the oracle's best within the logit tolerance
+            lg = res.logits[b]
+            tol = ROW_TOL * np.linalg.norm(lg, axis=1)
+            assert np.all(lg[np.arange(len(lm)), pred[b, lm]] >= lg.max(axis=1) - 2 * tol)
+        if len(S):
+            np.testing.assert_allclose(c[b], pair.ost.c[b], rtol=2e-2, atol=1e-4)
+
+
+def _prefill(pair):
+    g = pair.gpu_step(10 ** 6, 1.0, want_logits=True)
+    for b in range(pair.wl.batch):
+        assert g["sel"][b].tolist() == list(range(pair.wl.seq_len))
+    res = pair.oracle_step(g["sel"])
+    for b in range(pair.wl.batch):
+        assert row_rel_err(g["hidden"][b], res.hidden[b]) <= ROW_TOL
+    lg = np.concatenate(res.logits)
+    assert row_rel_err(g["logits"][: len(lg)], lg) <= ROW_TOL
+    _compare_state(pair, res, g["sel"])
+    return g, res
+
+
+WLS = {
+    "toy": inputs.WORKLOADS["toy"],
+    "gqa_bias_3layers": inputs.Workload("gqa", inputs.TOY_GQA, 2, 200, 120, 37, "random", 6, 0.7, seed=3),
+    "hd128_ragged_vocab": inputs.Workload("hd128", inputs.TOY_HD128, 3, 130, 70, 33, "random", 5, 0.5, seed=4),
+}
+
+
+@pytest.mark.parametrize("name", list(WLS))
+def test_prefill_then_partial_steps(name):
+    wl = WLS[name]
+    pair = Pair(wl)
+    _prefill(pair)
+    kc0 = pair.ctx.view("kcache").clone(); vc0 = pair.ctx.view("vcache").clone()
+    for step, (k, p) in enumerate([(wl.k, wl.p), (wl.k, 0.1), (3, 0.5)]):
+        g = pair.gpu_step(k, p, want_logits=True)
+        # bit-exact selection given the scores the GPU held before the step
+        want_sel = pair.oracle_selection(g["conf_before"], g["c_before"], pair.mask, k, p)
+        for b in range(wl.batch):
+            np.testing.assert_array_equal(g["sel"][b], want_sel[b], err_msg=f"step {step} seq {b}")
+            assert 0 < len(g["sel"][b]) < wl.seq_len
+        res = pair.oracle_step(g["sel"])
+        for b in range(wl.batch):
+            assert row_rel_err(g["hidden"][b], res.hidden[b]) <= ROW_TOL
+        _compare_state(pair, res, g["sel"])
+        # reuse: cache rows of unselected positions are bit-identical
+        kc1 = pair.ctx.view("kcache"); vc1 = pair.ctx.view("vcache")
+        for b in range(wl.batch):
+            rest = np.setdiff1d(np.arange(wl.seq_len), g["sel"][b])
+            assert torch.equal(kc1[:, b, rest], kc0[:, b, rest]) and torch.equal(vc1[:, b, rest], vc0[:, b, rest])
+        kc0, vc0 = kc1.clone(), vc1.clone()
+
+
+def test_single_layer_partial_step_reproduces_prefill_rows():
+    wl = WLS["toy"]
+    pair = Pair(wl)
+    g0, _ = _prefill(pair)
+    kc0 = pair.ctx.view("kcache").clone()
+    g = pair.gpu_step(wl.k, wl.p)
+    S = g["sel"][0]
+    assert len(S) < wl.seq_len
+    # with one layer nothing in the cache is stale, so the partial step recomputes the same values
+    assert row_rel_err(g["hidden"][0], g0["hidden"][0][S]) <= 1e-2
+    assert torch.equal(pair.ctx.view("kcache"), kc0)
+
+
+def test_select_none_changes_nothing():
+    pair = Pair(WLS["gqa_bias_3layers"])
+    _prefill(pair)
+    names = ("kcache", "vcache")
+    before = {n: pair.ctx.view(n).clone() for n in names}
+    B, L = pair.wl.batch, pair.wl.seq_len
+    sb = {n: pair.ctx.view(n, B, L).clone() for n in ("conf", "pred", "c")}
+    g = pair.gpu_step(0, 0.0)
+    assert g["row_off"].tolist() == [0] * (B + 1)
+    for n in names:
+        assert torch.equal(pair.ctx.view(n), before[n]), n
+    for n in sb:
+        assert torch.equal(pair.ctx.view(n, B, L), sb[n]), n
+
+
+def test_forced_rows_decoded_token_and_mode1():
+    wl = WLS["gqa_bias_3layers"]
+    pair = Pair(wl, stage2_candidates=1)
+    _prefill(pair)
+    # commit one token per sequence by hand: its embedding changes and it is forced into the next step
+    mask = pair.mask.clone(); h0 = pair.h0.clone(); forced = []
+    for b in range(wl.batch):
+        pos = int(np.flatnonzero(mask[b].numpy())[3])
+        mask[b, pos] = 0; h0[b, pos] = pair.w_cpu["embed"][17 + b]; forced.append([pos])
+    g = pair.gpu_step(4, 0.3, forced=forced, mask=mask, h0=h0, want_logits=True)
+    want_sel = pair.oracle_selection(g["conf_before"], g["c_before"], mask, 4, 0.3, forced=forced)
+    for b in range(wl.batch):
+        np.testing.assert_array_equal(g["sel"][b], want_sel[b])
+        assert forced[b][0] in g["sel"][b]
+    res = pair.oracle_step(g["sel"], mask=mask, h0=h0)
+    for b in range(wl.batch):
+        assert row_rel_err(g["hidden"][b], res.hidden[b]) <= ROW_TOL
+    _compare_state(pair, res, g["sel"], mask=mask)
+
+
+def test_step_is_deterministic():
+    wl = WLS["hd128_ragged_vocab"]
+    outs = []
+    for _ in range(2):
+        pair = Pair(wl)
+        pair.gpu_step(10 ** 6, 1.0)
+        g = pair.gpu_step(wl.k, wl.p)
+        outs.append((g, pair.ctx.view("c", wl.batch, wl.seq_len).clone(), pair.ctx.view("kcache").clone()))
+    for b in range(wl.batch):
+        np.testing.assert_array_equal(outs[0][0]["sel"][b], outs[1][0]["sel"][b])
+        np.testing.assert_array_equal(outs[0][0]["hidden"][b], outs[1][0]["hidden"][b])
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+
+
+def test_step_host_matches_device_step():
+    wl = WLS["toy"]
+    pair = Pair(wl)
+    pair.gpu_step(10 ** 6, 1.0)
+    B, L, d = wl.batch, wl.seq_len, wl.shape.d_model
+    snap = {n: pair.ctx.view(n, B, L).clone() for n in ("conf", "c")}
+    g = pair.gpu_step(wl.k, wl.p)
+    conf_dev = pair.ctx.view("conf", B, L).cpu()
+    for n, t in snap.items():
+        pair.ctx.view(n, B, L).copy_(t)
+    sel = torch.full((B * L,), -1, dtype=torch.int32).pin_memory(); ro = torch.zeros(B + 1, dtype=torch.int32).pin_memory()
+    hid = torch.zeros(B * L, d, dtype=torch.bfloat16).pin_memory()
+    conf = torch.zeros(B, L).pin_memory(); pred = torch.zeros(B, L, dtype=torch.int32).pin_memory()
+    pair.ctx.step_host(pair.h0.pin_memory(), pair.mask.pin_memory(), wl.k, wl.p, sel_idx=sel, row_off=ro, hidden_out=hid,
+                       conf=conf, pred=pred)
+    n = int(ro[B])
+    assert ro.numpy().tolist() == g["row_off"].tolist()
+    np.testing.assert_array_equal(sel.numpy()[:n], np.concatenate(g["sel"]))
+    np.testing.assert_array_equal(hid.float().numpy()[:n], np.concatenate(g["hidden"]))
+    assert torch.equal(conf, conf_dev)

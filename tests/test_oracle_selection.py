@@ -180,6 +180,11 @@ def test_stage2_ties_prefer_lower_positions_and_bad_scores_count_as_zero():
     c = np.array([np.nan, -1.0, 0.25, 0.75], dtype=np.float32)
     assert sel.stage2_select(c, cand, 0.5).tolist() == [3]
     assert sel.stage2_select(c, cand, 0.8).tolist() == [2, 3]
+    c = np.array([np.inf, -np.inf, 0.25, 0.75], dtype=np.float32)
+    assert sel.stage2_select(c, cand, 0.5).tolist() == [3]
+    c = np.array([1e30, 262144.0, 1.0, 1.0], dtype=np.float32)          # capped: the two large ones tie
+    assert sel.stage2_select(c, cand, 0.4).tolist() == [0]
+    assert sel.stage2_select(c, cand, 0.6).tolist() == [0, 1]
 
 
 def test_select_rows_union_and_candidate_modes():
