@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the d2Cache decode step (d2c_step) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole hot path (selection, gather, layers on the selected rows,
+LM head on the masked rows, rollout) over one batch of seeded synthetic input.  The default
+workload is one LLaDA-8B-shaped layer at sequence length 1024 (prefill, then the timed partial
+step with k=32, p=0.9).  Prints one JSON line.
+
+The path does not shard (one model replica per GPU, no exchange step): with --gpus N every rank
+runs an independent replica and the line reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_23094_b200 import inputs  # noqa: E402
+
+METRIC = "d2c_step selected tokens/s"
+UNIT = "selected_tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.file = index, None, None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        clocks, reasons, mx = [], set(), None
+        for line in self.file:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                clocks.append(float(parts[0])); mx = float(parts[1])
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks))
+        return out
+
+
+def algorithmic_work(shape, batch, L, n_b, n_m, rollout_layers):
+    """FLOPs and HBM bytes one step has to do (selected rows only; each weight read once)."""
+    n = sum(n_b)
+    P_l = shape.params_per_layer
+    N, d, Hq, Hkv, Dh, V = shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.vocab
+    flops = N * (2 * n * P_l + 4 * Hq * Dh * sum(nb * L for nb in n_b)) + 2 * n_m * d * V
+    byts = 2 * N * P_l + 2 * d * V
+    byts += N * sum(2 * L * Hkv * Dh * 2 + 2 * nb * Hkv * Dh * 2 for nb in n_b)
+    byts += 2 * n * d * 2
+    byts += rollout_layers * sum(2 * nb * L * 4 for nb in n_b)
+    return flops, byts
+
+
+def build_pair(wl, device):
+    from paper_2509_23094_b200 import binding
+    w_cpu = inputs.make_weights(wl.shape, seed=wl.seed, device=device if wl.shape.n_layers > 4 else "cpu")
+    w_dev = {"layers": [{k: (None if v is None else v.to(device)) for k, v in lyr.items()} for lyr in w_cpu["layers"]],
+             "g_final": w_cpu["g_final"].to(device), "w_lm": w_cpu["w_lm"].to(device), "embed": w_cpu["embed"].to(device)}
+    cfg = binding.make_config(wl.shape, wl.batch, wl.seq_len, sigma=wl.sigma)
+    ctx = binding.Context(cfg, w_dev, device=device)
+    mask = inputs.make_mask(wl)
+    tokens = inputs.make_tokens(wl, mask)
+    h0 = w_dev["embed"][tokens.to(device)].contiguous()
+    return w_cpu, w_dev, ctx, mask, tokens, h0
+
+
+def run_ours(args, rank, world, device):
+    wl = inputs.WORKLOADS[args.workload]
+    shape, B, L, d = wl.shape, wl.batch, wl.seq_len, wl.shape.d_model
+    w_cpu, w_dev, ctx, mask, tokens, h0 = build_pair(wl, device)
+    mask_dev = mask.to(device)
+    stream = torch.cuda.current_stream()
+
+    # prefill: every row, fills the cache, the confidences and the rollout scores
+    ctx.step(h0, mask_dev, 10 ** 6, 1.0)
+    ctx.sync_status()
+    snap = {n: ctx.view(n, B, L).clone() for n in ("conf", "pred", "c")}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)       # > L2 (126 MB)
+    hid = torch.zeros(B * L, d, dtype=torch.bfloat16, device=device)
+
+    def restore():
+        for n, t in snap.items():
+            ctx.view(n, B, L).copy_(t)
+        flush.fill_(1)
+
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    for _ in range(args.warmup):
+        restore()
+        ctx.step(h0, mask_dev, wl.k, wl.p, hidden_out=hid)
+    ctx.sync_status()
+    row_off = ctx.view("row_off", B, L).cpu().numpy()
+    lm_off = ctx.view("lm_off", B, L).cpu().numpy()
+    n_b = [int(row_off[b + 1] - row_off[b]) for b in range(B)]
+    n, n_m = int(row_off[B]), int(lm_off[B])
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    if world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ctx.profile(True)
+    ctx.profile_read(reset=True)
+    for i in range(args.steps):
+        restore()
+        ev0[i].record(stream)
+        ctx.step(h0, mask_dev, wl.k, wl.p, hidden_out=hid)
+        ev1[i].record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    clocks = sampler.stop()
+    phases = ctx.profile_read(reset=True)
+    ctx.profile(False)
+    ctx.sync_status()
+    per_step_ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+    total_ms = sum(per_step_ms)
+
+    # end to end: host buffers in, host results out, through d2c_step_host
+    h0_host = h0.cpu().pin_memory(); mask_host = mask.pin_memory()
+    sel_h = torch.empty(B * L, dtype=torch.int32).pin_memory(); ro_h = torch.empty(B + 1, dtype=torch.int32).pin_memory()
+    hid_h = torch.empty(B * L, d, dtype=torch.bfloat16).pin_memory()
+    conf_h = torch.empty(B, L).pin_memory(); pred_h = torch.empty(B, L, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_s = 0.0
+    for i in range(2 + e2e_steps):
+        restore()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ctx.step_host(h0_host, mask_host, wl.k, wl.p, sel_idx=sel_h, row_off=ro_h, hidden_out=hid_h, conf=conf_h, pred=pred_h)
+        if i >= 2:
+            e2e_s += time.perf_counter() - t0
+    h2d = B * L * d * 2 + B * L
+    d2h = (B + 1) * 4 + n * 4 + n * d * 2 + 2 * B * L * 4
+
+    # aggregate over ranks (independent replicas): max time, summed rows
+    t = torch.tensor([total_ms, e2e_s, float(n)], dtype=torch.float64, device=device)
+    if world > 1:
+        tmax = t.clone(); torch.distributed.all_reduce(tmax, op=torch.distributed.ReduceOp.MAX)
+        tsum = t.clone(); torch.distributed.all_reduce(tsum, op=torch.distributed.ReduceOp.SUM)
+        total_ms, e2e_s, n_all = float(tmax[0]), float(tmax[1]), float(tsum[2])
+    else:
+        n_all = float(n)
+    ms_per_step = total_ms / args.steps
+    value = n_all / (ms_per_step * 1e-3)
+    e2e_value = n_all / (e2e_s / e2e_steps)
+
+    peaks = measured_peaks()
+    depth = shape.n_layers
+    flops, byts = algorithmic_work(shape, B, L, n_b, n_m, depth)
+    t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
+    # dominant kernel: the projection / feed-forward GEMMs
+    gemm_ms = sum(phases[k]["ms"] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) / args.steps
+    gemm_launches = sum(phases[k]["launches"] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) // args.steps
+    gemm_flops = shape.n_layers * 2 * n * shape.params_per_layer
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    roofline = {"bound": "tensor", "kernel": "projection/FFN GEMMs (4 launches per layer)", "achieved": round(achieved, 2),
+                "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
+                "frac": round(achieved / peaks["bf16_tflops"], 4), "traffic": None,
+                "launches_per_step": int(gemm_launches), "ms_per_step": round(gemm_ms, 4),
+                "step_roofline_ms": round(t_roof * 1e3, 4), "step_frac": round(t_roof * 1e3 / ms_per_step, 4),
+                "step_flops": flops, "step_bytes": byts}
+    lm_ms = phases["lm_head"]["ms"] / args.steps
+    lm_bytes = 2 * d * shape.vocab
+    roofline["lm_head"] = {"bound": "hbm", "achieved": round(lm_bytes / (lm_ms * 1e-3) / 1e9, 1) if lm_ms > 0 else 0.0,
+                           "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                           "frac": round(lm_bytes / (lm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4) if lm_ms > 0 else 0.0,
+                           "ms_per_step": round(lm_ms, 4)}
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "shape": shape.name, "batch": B, "seq_len": L, "k": wl.k, "p": wl.p,
+                   "selected_rows": n_b, "lm_rows": n_m, "l2": "flushed between steps; weights (%.2f GB) exceed L2" %
+                   ((2 * shape.n_layers * shape.params_per_layer + 2 * d * shape.vocab) / 1e9),
+                   "replicas": world},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(e2e_s / e2e_steps * 1e3, 4)},
+        "gpu_launches": int(sum(p["launches"] for p in phases.values())),
+        "roofline": roofline,
+        "phases_ms_per_step": {k: round(v["ms"] / args.steps, 4) for k, v in phases.items()},
+        "step_ms_min": round(min(per_step_ms), 4), "step_ms_median": round(statistics.median(per_step_ms), 4),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L)
+    return line
+
+
+def oracle_setup(wl, w_cpu, mask, tokens):
+    from oracle import step as ostep
+    wf = ostep.weights_to_f64(w_cpu)
+    h0 = inputs.make_h0(w_cpu["embed"].cpu(), tokens).double().numpy()
+    st = ostep.OracleState(wl.shape.n_layers, wl.batch, wl.seq_len, wl.shape.n_kv_heads, wl.shape.head_dim)
+    return ostep, wf, h0, st
+
+
+def cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L, max_rows=256):
+    """The oracle, as it stands, on the host cores: one partial step on a bounded sample of the rows."""
+    if wl.shape.n_layers > 4:
+        return {"value": None, "unit": UNIT, "kind": "oracle", "cores": os.cpu_count(),
+                "sample": "skipped: the full-depth model does not fit the CPU time budget"}
+    ostep, wf, h0, st = oracle_setup(wl, w_cpu, mask, tokens)
+    row_off = ctx.view("row_off", B, L).cpu().numpy()
+    sel = ctx.view("sel_idx").cpu().numpy()
+    # the cache the sampled rows attend to: taken from a full oracle forward of layer inputs would cost
+    # a prefill; the timing only needs a cache of the right shape, so it is filled with random values
+    rng = np.random.default_rng(0)
+    st.Kc[:] = rng.standard_normal(st.Kc.shape) * 0.1
+    st.Vc[:] = rng.standard_normal(st.Vc.shape) * 0.1
+    sample = []
+    for b in range(B):
+        S = sel[row_off[b]: row_off[b + 1]].astype(np.int64)
+        take = max(1, max_rows // B)
+        sample.append(S[:: max(1, len(S) // take)][:take])
+    rows = sum(len(s) for s in sample)
+    t0 = time.perf_counter()
+    ostep.oracle_step(st, wf, wl.shape, h0, mask.numpy(), k=0, p=0.0, sigma=wl.sigma, sel_override=sample)
+    dt = time.perf_counter() - t0
+    return {"value": round(rows / dt, 2), "unit": UNIT, "kind": "oracle", "cores": os.cpu_count(),
+            "sample": f"one oracle step on {rows} of the selected rows (fp64 numpy), {dt:.1f} s"}
+
+
+def run_reference(args):
+    """Times the oracle on the host cores; each step is one partial step on a bounded sample of rows."""
+    wl = inputs.WORKLOADS[args.workload]
+    if wl.shape.n_layers > 4:
+        print(json.dumps({"impl": "reference", "unavailable": "the full-depth workload does not fit the CPU time budget"}))
+        return
+    B, L = wl.batch, wl.seq_len
+    w_cpu = inputs.make_weights(wl.shape, seed=wl.seed)
+    mask = inputs.make_mask(wl)
+    tokens = inputs.make_tokens(wl, mask)
+    ostep, wf, h0, st = oracle_setup(wl, w_cpu, mask, tokens)
+    rng = np.random.default_rng(0)
+    st.Kc[:] = rng.standard_normal(st.Kc.shape) * 0.1
+    st.Vc[:] = rng.standard_normal(st.Vc.shape) * 0.1
+    st.conf[:] = rng.random(st.conf.shape).astype(np.float32)
+    st.c[:] = (1.0 + 0.05 * rng.standard_normal(st.c.shape)).astype(np.float32)
+    from oracle import selection as osel
+    rows_per_step = 96
+    sample = []
+    for b in range(B):
+        S, _, _ = osel.select_rows(mask[b].numpy(), st.conf[b], st.c[b], wl.k, wl.p, wl.sigma)
+        take = max(1, rows_per_step // B)
+        sample.append(S[:: max(1, len(S) // take)][:take])
+    rows = sum(len(s) for s in sample)
+    snap_conf, snap_c = st.conf.copy(), st.c.copy()
+    times = []
+    for i in range(args.warmup + args.steps):
+        st.conf[:] = snap_conf; st.c[:] = snap_c
+        t0 = time.perf_counter()
+        ostep.oracle_step(st, wf, wl.shape, h0, mask.numpy(), k=0, p=0.0, sigma=wl.sigma, sel_override=sample)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    ms = 1e3 * sum(times) / len(times)
+    value = rows / (ms * 1e-3)
+    desc = f"each step: one oracle step on {rows} of the selected rows (fp64 numpy)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "shape": wl.shape.name, "batch": B, "seq_len": L, "k": wl.k, "p": wl.p},
+        "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "kind": "oracle", "cores": os.cpu_count(), "sample": desc},
+        "e2e": {"value": round(value, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="llada1l_1024", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=torch.device(device))
+    line = run_ours(args, rank, world, device)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

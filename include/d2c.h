@@ -65,8 +65,9 @@ typedef struct {
   int32_t stage2_candidates;  /* 0: top-p runs over known (prompt/decoded) positions;
                                  1: over every position stage 1 did not take                             */
   int32_t rollout_layers;     /* 0: rollout over all layers (Eq. 8); n>0: only the first n layers        */
-  int32_t flags;              /* reserved, must be 0                                                     */
+  int32_t flags;              /* D2C_FLAG_* bits                                                         */
 } d2c_config;
+#define D2C_FLAG_PORTABLE_GEMM 1   /* run the GEMMs on the mma.sync kernel instead of the tcgen05 one (cross-check) */
 
 /* Weights.  The arrays of per-layer pointers are HOST arrays of n_layers DEVICE
  * pointers; they are copied at create, the device memory is borrowed for the
@@ -161,10 +162,24 @@ typedef struct {
   float*   lse;         /* f32 [max_batch*max_seq][Hq] log-sum-exp of the last layer's scores        */
   int32_t* status;      /* [4] device status word: [0] error code, [1] where                         */
 } d2c_state;
+/* The per-position vectors (conf, pred, c, key) are indexed [b*seq_len + pos] with the batch and
+ * seq_len of the d2c_step calls; a context is used with one (batch, seq_len) from its first step on.
+ * abar: row r of layer l is at abar + l*max_batch*max_seq*max_seq + r*seq_len. */
 int d2c_state_ptrs(d2c_ctx* ctx, d2c_state* out);
 
 /* Synchronises the stream and returns the device status word's error code. */
 int d2c_sync_status(d2c_ctx* ctx);
+
+/* Per-phase timing of d2c_step.  While enabled, d2c_step records one CUDA event at every phase
+ * boundary on the context's stream (events are host objects; no device memory is allocated).
+ * d2c_profile_read synchronises the stream and returns, accumulated since the last reset, the
+ * milliseconds spent in each phase (phase_ms[D2C_N_PHASES]) and the number of kernels the library
+ * launched in it (phase_launches[D2C_N_PHASES]); either may be NULL.  d2c_phase_name(i) names
+ * phase i ("select", "gemm_qkv", ...). */
+#define D2C_N_PHASES 12
+int d2c_profile(d2c_ctx* ctx, int32_t enable);
+int d2c_profile_read(d2c_ctx* ctx, float* phase_ms, int64_t* phase_launches, int32_t reset);
+const char* d2c_phase_name(int32_t i);
 
 /* Text of the last error on this context (host string, never NULL); with ctx == NULL the
  * last error of a failed d2c_create / stand-alone op on this thread. */

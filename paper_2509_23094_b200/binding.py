@@ -14,11 +14,12 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libd2c.so")
 
+N_PHASES = 12
 D2C_OK, D2C_EINVAL, D2C_ESHAPE, D2C_ECAPACITY, D2C_ECUDA, D2C_ETIMEOUT = 0, -1, -2, -3, -4, -5
 
 # every symbol include/d2c.h declares
 SYMBOLS = ["d2c_workspace_bytes", "d2c_create", "d2c_step", "d2c_step_host", "d2c_commit", "d2c_state_ptrs",
-           "d2c_sync_status", "d2c_last_error", "d2c_destroy", "d2c_op_select_scratch_bytes", "d2c_op_select",
+           "d2c_sync_status", "d2c_last_error", "d2c_destroy", "d2c_profile", "d2c_profile_read", "d2c_phase_name", "d2c_op_select_scratch_bytes", "d2c_op_select",
            "d2c_op_gemm", "d2c_op_attention", "d2c_op_lm_head_scratch_bytes", "d2c_op_lm_head",
            "d2c_op_rollout_scratch_bytes", "d2c_op_rollout"]
 
@@ -84,6 +85,10 @@ def load() -> C.CDLL:
     lib.d2c_last_error.restype = C.c_char_p
     lib.d2c_last_error.argtypes = [vp]
     lib.d2c_destroy.argtypes = [vp]
+    lib.d2c_profile.argtypes = [vp, i32]
+    lib.d2c_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64), i32]
+    lib.d2c_phase_name.restype = C.c_char_p
+    lib.d2c_phase_name.argtypes = [i32]
     lib.d2c_op_select_scratch_bytes.restype = sz
     lib.d2c_op_select_scratch_bytes.argtypes = [i32, i32]
     lib.d2c_op_select.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -125,10 +130,10 @@ def _check(rc: int, ctx: Optional[int] = None) -> None:
 
 
 def make_config(shape, max_batch: int, max_seq: int, sigma: float = 10.0, stage2_candidates: int = 0,
-                rollout_layers: int = 0) -> Config:
+                rollout_layers: int = 0, flags: int = 0) -> Config:
     return Config(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
                   shape.vocab, max_batch, max_seq, shape.rope_base, shape.rms_eps, sigma, int(shape.qkv_bias),
-                  stage2_candidates, rollout_layers, 0)
+                  stage2_candidates, rollout_layers, flags)
 
 
 def d2c_workspace_bytes(cfg: Config) -> int:
@@ -233,6 +238,16 @@ class Context:
         B, L = mask.shape
         _check(load().d2c_commit(self.handle, B, L, _ptr(embed), _ptr(h0), _ptr(mask), _ptr(tokens), _ptr(committed),
                                  int(rule), float(threshold)), self.handle)
+
+    def profile(self, enable: bool) -> None:
+        _check(load().d2c_profile(self.handle, int(enable)), self.handle)
+
+    def profile_read(self, reset: bool = True) -> Dict[str, Dict[str, float]]:
+        lib = load()
+        ms = (C.c_float * N_PHASES)()
+        ln = (C.c_int64 * N_PHASES)()
+        _check(lib.d2c_profile_read(self.handle, ms, ln, int(reset)), self.handle)
+        return {lib.d2c_phase_name(i).decode(): {"ms": float(ms[i]), "launches": int(ln[i])} for i in range(N_PHASES)}
 
     def sync_status(self) -> None:
         _check(load().d2c_sync_status(self.handle), self.handle)

@@ -256,10 +256,10 @@ int launch_dh(const AttnArgs& a, cudaStream_t st) {
   }
   const int qtiles = ceil_div(a.max_rows_per_seq, QT);
   attn_fwd_kernel<DH><<<dim3(qtiles, a.hq, a.batch), ATHREADS, smem_fwd, st>>>(a);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   if (a.abar) {
     attn_abar_kernel<DH><<<dim3(ceil_div(a.seq_len, KT), qtiles, a.batch), ATHREADS, smem_ab, st>>>(a);
-    D2C_CUDA_OK(cudaGetLastError());
+    D2C_LAUNCHED();
   }
   return D2C_OK;
 }

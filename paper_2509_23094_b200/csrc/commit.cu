@@ -65,7 +65,7 @@ int launch_commit(int batch, int seq_len, int d, int rule, float threshold, cons
                   bf16* h0, uint8_t* mask, int32_t* tokens, int32_t* committed, cudaStream_t st) {
   CommitArgs a{seq_len, d, rule, threshold, slot_of_pos, conf, pred, phi, phi_len, embed, h0, mask, tokens, committed};
   commit_kernel<<<batch, 256, seq_len, st>>>(a);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 

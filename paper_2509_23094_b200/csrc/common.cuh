@@ -16,6 +16,8 @@ namespace d2c {
 // Text of the last error raised outside any context (thread local).
 void set_global_error(const char* fmt, ...);
 const char* global_error();
+// Adds n to this thread's count of kernels launched by the library.
+void count_launch(int n);
 
 #define D2C_CUDA_OK(expr)                                                              \
   do {                                                                                 \
@@ -26,6 +28,8 @@ const char* global_error();
       return D2C_ECUDA;                                                                \
     }                                                                                  \
   } while (0)
+// After a kernel launch: checks the launch and counts it.
+#define D2C_LAUNCHED() do { D2C_CUDA_OK(cudaGetLastError()); d2c::count_launch(1); } while (0)
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -97,5 +101,6 @@ int launch_commit(int batch, int seq_len, int d, int rule, float threshold, cons
                   const float* conf, const int32_t* pred, const uint32_t* phi, int phi_len, const bf16* embed,
                   bf16* h0, uint8_t* mask, int32_t* tokens, int32_t* committed, cudaStream_t st);
 // ---- tcgen05 GEMM (gemm_tc.cu) -------------------------------------------------------------------
-int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st);
+// status: device int[4] that receives D2C_ETIMEOUT if a bounded wait runs out (null: a library-owned word).
+int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status = nullptr);
 }  // namespace d2c

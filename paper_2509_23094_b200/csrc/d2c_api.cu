@@ -17,6 +17,14 @@ void set_global_error(const char* fmt, ...) {
 }
 const char* global_error() { return g_err; }
 
+static thread_local long long g_launches = 0;
+void count_launch(int n) { g_launches += n; }
+
+static const char* const kPhaseNames[D2C_N_PHASES] = {
+    "select", "gather_norm", "rmsnorm", "gemm_qkv", "rope_scatter", "attention", "gemm_o",
+    "gemm_gate_up", "gemm_down", "lm_head", "rollout", "copy_out"};
+enum Phase { PH_SELECT = 0, PH_GATHER, PH_NORM, PH_QKV, PH_ROPE, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM, PH_ROLLOUT, PH_OUT };
+
 // Hands out 256-byte aligned pieces of a buffer; with base == null it only measures.
 struct Carver {
   char* base; size_t off = 0;
@@ -84,7 +92,7 @@ static const char* check_config(const d2c_config* c) {
   if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
   if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
   if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
-  if (c->rollout_layers < 0 || c->flags != 0) return "rollout_layers >= 0 and flags == 0 required";
+  if (c->rollout_layers < 0 || (c->flags & ~D2C_FLAG_PORTABLE_GEMM)) return "rollout_layers >= 0 and no unknown flag bits required";
   return nullptr;
 }
 
@@ -100,7 +108,32 @@ struct d2c_ctx {
   Buffers buf;
   int phi_len;
   char err[512];
+  // optional per-phase timing: one event at every phase boundary, resolved by d2c_profile_read
+  bool prof = false;
+  std::vector<cudaEvent_t> ev;
+  std::vector<int> ev_phase;      // phase that starts at event i, -1 = end of a step
+  size_t ev_used = 0;
+  double phase_ms[D2C_N_PHASES] = {0};
+  long long phase_launches[D2C_N_PHASES] = {0};
+  long long launch_mark = 0;
+  int prof_phase = -1;
 };
+
+// Marks the start of `phase` (or the end of the step with phase < 0) on the context's stream.
+static int mark(d2c_ctx* ctx, int phase) {
+  if (!ctx->prof) return D2C_OK;
+  if (ctx->prof_phase >= 0) ctx->phase_launches[ctx->prof_phase] += g_launches - ctx->launch_mark;
+  ctx->launch_mark = g_launches; ctx->prof_phase = phase;
+  if (ctx->ev_used == ctx->ev.size()) {
+    cudaEvent_t e;
+    D2C_CUDA_OK(cudaEventCreate(&e));
+    ctx->ev.push_back(e); ctx->ev_phase.push_back(-1);
+  }
+  ctx->ev_phase[ctx->ev_used] = phase;
+  D2C_CUDA_OK(cudaEventRecord(ctx->ev[ctx->ev_used], ctx->stream));
+  ctx->ev_used++;
+  return D2C_OK;
+}
 
 static int fail(d2c_ctx* ctx, int code, const char* fmt, ...) {
   char tmp[512];
@@ -113,6 +146,11 @@ static int fail(d2c_ctx* ctx, int code, const char* fmt, ...) {
 static int pass(d2c_ctx* ctx, int rc) {
   if (rc != D2C_OK && ctx) { strncpy(ctx->err, global_error(), sizeof(ctx->err) - 1); ctx->err[sizeof(ctx->err) - 1] = 0; }
   return rc;
+}
+// The step's GEMMs: tcgen05 kernel unless the context was created with D2C_FLAG_PORTABLE_GEMM.
+static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
+  if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->stream);
+  return launch_gemm_tc(g, epi, ctx->stream, ctx->buf.status);
 }
 #define D2C_TRY(ctx, expr) do { int rc__ = (expr); if (rc__ != D2C_OK) return pass((ctx), rc__); } while (0)
 
@@ -170,6 +208,7 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
 
 int d2c_destroy(d2c_ctx* ctx) {
   if (!ctx) return D2C_EINVAL;
+  for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   delete ctx;
   return D2C_OK;
 }
@@ -228,51 +267,66 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   s.stage2_candidates = c.stage2_candidates; s.phi_q30 = b.phi; s.phi_len = ctx->phi_len < L ? ctx->phi_len : L;
   s.key = b.key; s.sel_idx = b.sel_idx; s.row_seq = b.row_seq; s.row_off = b.row_off; s.lm_rows = b.lm_rows;
   s.lm_off = b.lm_off; s.slot_of_pos = b.slot_of_pos; s.rank_s = b.rank_s; s.rank_lm = b.rank_lm; s.n_b = b.n_b; s.nm_b = b.nm_b;
+  D2C_TRY(ctx, mark(ctx, PH_SELECT));
   D2C_TRY(ctx, launch_select(s, st));
   const int32_t* n_rows = b.row_off + B;
   const int32_t* n_lm = b.lm_off + B;
 
+  D2C_TRY(ctx, mark(ctx, PH_GATHER));
   D2C_TRY(ctx, launch_gather_norm((const bf16*)a->h0, b.sel_idx, b.row_seq, n_rows, R, L, d, ctx->g_attn[0], c.rms_eps, x, b.xn, st));
   const int depth = rollout_depth(c);
   for (int l = 0; l < c.n_layers; ++l) {
-    if (l > 0) D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
+    if (l > 0) {
+      D2C_TRY(ctx, mark(ctx, PH_NORM));
+      D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
+    }
+    D2C_TRY(ctx, mark(ctx, PH_QKV));
     GemmArgs g{};
     g.A = b.xn; g.lda = d; g.W = ctx->wqkv[l]; g.bias = ctx->bqkv[l]; g.C = b.qkv; g.ldc = qkv_out;
     g.n_rows = n_rows; g.max_rows = R; g.N = qkv_out; g.K = d;
-    D2C_TRY(ctx, launch_gemm_mma(g, EPI_STORE, st));
+    D2C_TRY(ctx, gemm(ctx, g, EPI_STORE));
     bf16* kc = b.kcache + (size_t)l * cache_layer; bf16* vc = b.vcache + (size_t)l * cache_layer;
+    D2C_TRY(ctx, mark(ctx, PH_ROPE));
     D2C_TRY(ctx, launch_rope_scatter(b.qkv, b.sel_idx, b.row_seq, n_rows, R, hq, hkv, dh, b.rope, kc, vc, c.max_seq, st));
     AttnArgs at{};
     at.q = b.qkv; at.ldq = qkv_out; at.kc = kc; at.vc = vc; at.row_off = b.row_off; at.batch = B; at.seq_len = L;
     at.cache_seq = c.max_seq; at.hq = hq; at.hkv = hkv; at.dh = dh; at.max_rows_per_seq = L;
     at.o = b.o; at.lse = b.lse; at.abar = l < depth ? b.abar + (size_t)l * c.max_batch * c.max_seq * c.max_seq : nullptr;
+    D2C_TRY(ctx, mark(ctx, PH_ATTN));
     D2C_TRY(ctx, launch_attention(at, st));
+    D2C_TRY(ctx, mark(ctx, PH_O));
     GemmArgs go{};
     go.A = b.o; go.lda = hq * dh; go.W = ctx->wo[l]; go.C = x; go.ldc = d; go.n_rows = n_rows; go.max_rows = R; go.N = d; go.K = hq * dh;
-    D2C_TRY(ctx, launch_gemm_mma(go, EPI_RESIDUAL, st));
+    D2C_TRY(ctx, gemm(ctx, go, EPI_RESIDUAL));
+    D2C_TRY(ctx, mark(ctx, PH_NORM));
     D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_ffn[l], c.rms_eps, b.xn, st));
+    D2C_TRY(ctx, mark(ctx, PH_GATEUP));
     GemmArgs gf{};
     gf.A = b.xn; gf.lda = d; gf.W = ctx->w_gate[l]; gf.W2 = ctx->w_up[l]; gf.C = b.hmid; gf.ldc = c.d_ffn;
     gf.n_rows = n_rows; gf.max_rows = R; gf.N = c.d_ffn; gf.K = d;
-    D2C_TRY(ctx, launch_gemm_mma(gf, EPI_SWIGLU, st));
+    D2C_TRY(ctx, gemm(ctx, gf, EPI_SWIGLU));
     GemmArgs gd{};
     gd.A = b.hmid; gd.lda = c.d_ffn; gd.W = ctx->w_down[l]; gd.C = x; gd.ldc = d; gd.n_rows = n_rows; gd.max_rows = R; gd.N = d; gd.K = c.d_ffn;
-    D2C_TRY(ctx, launch_gemm_mma(gd, EPI_RESIDUAL, st));
+    D2C_TRY(ctx, mark(ctx, PH_DOWN));
+    D2C_TRY(ctx, gemm(ctx, gd, EPI_RESIDUAL));
   }
   // Eq. 1 on the selected rows that are still masked
+  D2C_TRY(ctx, mark(ctx, PH_LM));
   D2C_TRY(ctx, launch_rmsnorm(x, b.lm_rows, n_lm, R, d, ctx->g_final, c.rms_eps, b.xm, st));
   GemmArgs gl{};
   gl.A = b.xm; gl.lda = d; gl.W = ctx->w_lm; gl.n_rows = n_lm; gl.max_rows = R; gl.N = c.vocab; gl.K = d;
   gl.st_max = b.st_max; gl.st_sum = b.st_sum; gl.st_arg = b.st_arg; gl.n_tiles = lm_tiles(c.vocab);
   gl.logits = out ? out->logits : nullptr;
-  D2C_TRY(ctx, launch_gemm_mma(gl, EPI_LMSTATS, st));
+  D2C_TRY(ctx, gemm(ctx, gl, EPI_LMSTATS));
   D2C_TRY(ctx, launch_lm_reduce(b.st_max, b.st_sum, b.st_arg, gl.n_tiles, n_lm, R, b.lm_rows, b.sel_idx, b.row_seq, L, b.conf, b.pred, st));
   // Eq. 6-9 for the next step's stage 2
+  D2C_TRY(ctx, mark(ctx, PH_ROLLOUT));
   RolloutArgs r{};
   r.abar = b.abar; r.layer_stride = (size_t)c.max_batch * c.max_seq * c.max_seq; r.n_layers = depth; r.sel_idx = b.sel_idx;
   r.row_off = b.row_off; r.batch = B; r.seq_len = L; r.c = b.c; r.u0 = b.u0; r.u1 = b.u1; r.partial = b.partial; r.n_split = kRolloutSplit;
   D2C_TRY(ctx, launch_rollout(r, st));
 
+  D2C_TRY(ctx, mark(ctx, PH_OUT));
   if (out && out->sel_idx) {
     cudaError_t e = cudaMemcpyAsync(out->sel_idx, b.sel_idx, (size_t)R * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
     if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
@@ -281,8 +335,38 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     cudaError_t e = cudaMemcpyAsync(out->row_off, b.row_off, (size_t)(B + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
     if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
   }
+  D2C_TRY(ctx, mark(ctx, -1));
   return D2C_OK;
 }
+
+int d2c_profile(d2c_ctx* ctx, int32_t enable) {
+  if (!ctx) return D2C_EINVAL;
+  ctx->prof = enable != 0;
+  ctx->prof_phase = -1;
+  return D2C_OK;
+}
+
+int d2c_profile_read(d2c_ctx* ctx, float* phase_ms, int64_t* phase_launches, int32_t reset) {
+  if (!ctx) return D2C_EINVAL;
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_profile_read: %s", cudaGetErrorString(e));
+  for (size_t i = 0; i + 1 < ctx->ev_used; ++i) {
+    if (ctx->ev_phase[i] < 0) continue;
+    float ms = 0.f;
+    e = cudaEventElapsedTime(&ms, ctx->ev[i], ctx->ev[i + 1]);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_profile_read: %s", cudaGetErrorString(e));
+    ctx->phase_ms[ctx->ev_phase[i]] += ms;
+  }
+  ctx->ev_used = 0;
+  for (int i = 0; i < D2C_N_PHASES; ++i) {
+    if (phase_ms) phase_ms[i] = (float)ctx->phase_ms[i];
+    if (phase_launches) phase_launches[i] = ctx->phase_launches[i];
+    if (reset) { ctx->phase_ms[i] = 0; ctx->phase_launches[i] = 0; }
+  }
+  return D2C_OK;
+}
+
+const char* d2c_phase_name(int32_t i) { return (i >= 0 && i < D2C_N_PHASES) ? kPhaseNames[i] : ""; }
 
 int d2c_step_host(d2c_ctx* ctx, const d2c_step_args* h, const d2c_host_out* out) {
   D2C_TRY(ctx, check_step_args(ctx, h));

@@ -231,7 +231,7 @@ int launch_one(const GemmArgs& g, cudaStream_t st) {
   const int n_tiles = EPI == EPI_SWIGLU ? ceil_div(g.N, 64) : ceil_div(g.N, BN);
   dim3 grid(n_tiles, ceil_div(g.max_rows, BM));
   gemm_mma_kernel<EPI><<<grid, THREADS, smem, st>>>(g);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 }  // namespace

@@ -1,8 +1,406 @@
-// tcgen05 / TMEM GEMM (placeholder until the kernel lands): reports that it is not built.
+// tcgen05 / TMEM GEMM for sm_100a with the step's fused epilogues.
+//
+//   C[m][n] = sum_k A[m][k] * W[n][k]      A: [max_rows][K] bf16, W: [N][K] bf16 (both K-major)
+//
+// One CTA computes one 128 x BN output tile (BN = 128, or 128 gate + 128 up columns for the SwiGLU
+// epilogue).  Warp roles:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of 128 x 64 bf16 boxes (128-byte swizzle) into a
+//               ring of shared-memory stages, completion signalled on mbarriers;
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared-memory
+//               descriptors into a TMEM accumulator; tcgen05.commit releases each stage back to the
+//               producer and finally signals the epilogue;
+//   warps 2-5   epilogue: tcgen05.ld brings one accumulator row per thread into registers, the fused
+//               epilogue (bias / residual / SwiGLU / soft-max statistics) runs there, rows go to HBM.
+// The live row count is read from device memory: tiles past it exit before allocating anything.
+// Every mbarrier wait is bounded; a wait that runs out raises D2C_ETIMEOUT in the status word, the
+// CTA drains its copies, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace d2c {
-int launch_gemm_tc(const GemmArgs&, GemmEpilogue, cudaStream_t) {
-  set_global_error("tcgen05 GEMM is not built in this library");
-  return D2C_ESHAPE;
+namespace {
+
+constexpr int TM = 128, TK = 64;                 // tile rows, K elements per stage (one 128-byte swizzle atom)
+constexpr int TC_THREADS = 192;
+constexpr int A_BYTES = TM * TK * 2;             // 16 KB
+constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
+
+__device__ int g_tc_status[4];                   // status word used when the caller passes none
+
+// ------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile("{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
+               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done;
+}
+// Bounded wait.  Returns false if it gave up (or another thread of the CTA already had).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = site;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                 "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                 "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                 "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte rows with the 128-byte
+// swizzle (what the TMA box load produces): 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);      // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+
+union Pack8 { uint4 u; __nv_bfloat162 h[4]; };
+
+struct TcParams {
+  GemmArgs g;
+  int* status;
+  int stages;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  constexpr int BN = (EPI == EPI_SWIGLU) ? 256 : 128;        // accumulator columns
+  constexpr int B_BYTES = BN * TK * 2;
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int OUT_COLS = 128;                              // output columns per tile
+  const GemmArgs& g = p.g;
+  const int n = *g.n_rows;
+  const int m0 = blockIdx.y * TM;
+  if (m0 >= n) return;                                       // uniform: nothing allocated yet
+  const int n0 = blockIdx.x * OUT_COLS;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KT = g.K / TK, ST = p.stages;
+  int* status = p.status ? p.status : g_tc_status;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
+  __shared__ __align__(8) uint64_t bars[2 * 8 + 1];          // full[ST], empty[ST], accumulator-ready
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
+  const uint32_t acc_bar = bar0 + 8u * 16;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_slot;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int issued = 0;
+      for (int kt = 0; kt < KT; ++kt) {
+        const int s = kt % ST;
+        const uint32_t parity = ((kt / ST) & 1) ^ 1;          // a fresh barrier passes a wait on parity 1
+        if (!mbar_wait(empty_bar(s), parity, abortp, status, 1)) break;
+        const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+        tma_load_2d(sa, &tmA, kt * TK, m0, full_bar(s));
+        tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
+        if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
+        issued = kt + 1;
+      }
+      if (*abortp) {
+        // give the copies already in flight a bounded chance to land before the CTA goes away
+        for (int kt = max(0, issued - ST); kt < issued; ++kt) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full_bar(kt % ST), (kt / ST) & 1) && clock64() - t0 < kWaitCycles) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(BN);
+      bool ok = true;
+      for (int kt = 0; kt < KT && ok; ++kt) {
+        const int s = kt % ST;
+        ok = mbar_wait(full_bar(s), (kt / ST) & 1, abortp, status, 2);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+        const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k)                     // +32 bytes per K=16 slice inside the swizzle atom
+          umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+        umma_commit(empty_bar(s));                            // stage reusable once these MMAs have read it
+      }
+      if (ok) umma_commit(acc_bar);                           // accumulator complete
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                             // TMEM lanes this warp may touch
+    const int lrow = quarter * 32 + lane;
+    const int row = m0 + lrow;
+    const bool row_ok = row < n;
+    const bool ready = mbar_wait(acc_bar, 0, abortp, status, 3);
+    tc_fence_after();
+    if (ready) {
+      const uint32_t tbase = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+      if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+        const bool vec = (g.ldc & 7) == 0;
+#pragma unroll 1
+        for (int c = 0; c < OUT_COLS / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tbase + c * 32, v);
+          tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if (!row_ok || col0 >= g.N) continue;
+          bf16* dst = g.C + (size_t)row * g.ldc + col0;
+          if (vec && col0 + 32 <= g.N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              Pack8 o, old;
+              if (EPI == EPI_RESIDUAL) old.u = reinterpret_cast<const uint4*>(dst)[q];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
+                if (EPI == EPI_STORE) {
+                  if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
+                } else {
+                  const float2 of = __bfloat1622float2(old.h[e]);
+                  f0 += of.x; f1 += of.y;
+                }
+                o.h[e] = __floats2bfloat162_rn(f0, f1);
+              }
+              reinterpret_cast<uint4*>(dst)[q] = o.u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (col0 + j < g.N) {
+                float f = __uint_as_float(v[j]);
+                if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
+                else f += __bfloat162float(dst[j]);
+                dst[j] = __float2bfloat16_rn(f);
+              }
+            }
+          }
+        }
+      } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < OUT_COLS / 32; ++c) {
+          uint32_t gv[32], uv[32];
+          tmem_ld32(tbase + c * 32, gv);
+          tmem_ld32(tbase + 128 + c * 32, uv);
+          tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if (!row_ok || col0 >= g.N) continue;
+          bf16* dst = g.C + (size_t)row * g.ldc + col0;
+          if ((g.ldc & 7) == 0 && col0 + 32 <= g.N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              Pack8 o;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float g0 = __uint_as_float(gv[q * 8 + 2 * e]), g1 = __uint_as_float(gv[q * 8 + 2 * e + 1]);
+                const float u0 = __uint_as_float(uv[q * 8 + 2 * e]), u1 = __uint_as_float(uv[q * 8 + 2 * e + 1]);
+                o.h[e] = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+              }
+              reinterpret_cast<uint4*>(dst)[q] = o.u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (col0 + j < g.N) {
+                const float gg = __uint_as_float(gv[j]), uu = __uint_as_float(uv[j]);
+                dst[j] = __float2bfloat16_rn(gg / (1.f + __expf(-gg)) * uu);
+              }
+            }
+          }
+        }
+      } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
+        float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
+#pragma unroll 1
+        for (int c = 0; c < OUT_COLS / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tbase + c * 32, v);
+          tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if (col0 >= g.N) continue;
+          float cmx = -INFINITY; int carg = 0x7fffffff;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float f = __uint_as_float(v[j]);
+            if (col0 + j < g.N && f > cmx) { cmx = f; carg = col0 + j; }     // ascending columns: first maximum wins
+          }
+          const float nmx = fmaxf(mx, cmx);
+          float csum = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < g.N) csum += __expf(__uint_as_float(v[j]) - nmx);
+          sum = sum * __expf(mx - nmx) + csum;                                // exp(-inf) = 0 on the first chunk
+          if (cmx > mx) arg = carg;
+          mx = nmx;
+          if (g.logits && row_ok) {
+            float* lp = g.logits + (size_t)row * g.N + col0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < g.N) lp[j] = __uint_as_float(v[j]);
+          }
+        }
+        if (row_ok) {
+          const size_t o = (size_t)row * g.n_tiles + blockIdx.x;
+          g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
+        }
+      }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_acc, BN);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D map over a row-major bf16 matrix [rows][cols] with leading dimension ld; box = 128 rows x 64 columns,
+// 128-byte swizzle, out-of-range elements read as zero.
+int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_global_error("cuTensorMapEncodeTiled is not available from this driver"); return D2C_ECUDA; }
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {TK, TM};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_global_error("cuTensorMapEncodeTiled failed with code %d", (int)r); return D2C_ECUDA; }
+  return D2C_OK;
+}
+
+template <int EPI>
+int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
+  constexpr int BN = (EPI == EPI_SWIGLU) ? 256 : 128;
+  constexpr int STAGE_BYTES = A_BYTES + BN * TK * 2;
+  const int stages = (EPI == EPI_SWIGLU) ? 4 : 6;
+  const int smem = stages * STAGE_BYTES + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB, tmB2;
+  int rc = make_map(&tmA, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda);
+  if (rc != D2C_OK) return rc;
+  rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K);
+  if (rc != D2C_OK) return rc;
+  rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K);
+  if (rc != D2C_OK) return rc;
+  TcParams p{g, status, stages};
+  dim3 grid(ceil_div(g.N, 128), ceil_div(g.max_rows, TM));
+  gemm_tc_kernel<EPI><<<grid, TC_THREADS, smem, st>>>(tmA, tmB, tmB2, p);
+  D2C_LAUNCHED();
+  return D2C_OK;
+}
+}  // namespace
+
+int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status) {
+  if (g.max_rows <= 0 || g.N <= 0) return D2C_OK;
+  // shapes the TMA boxes cannot express fall back to the portable kernel
+  if (g.max_rows < TM || g.N < 128 || g.K % TK != 0 || (g.lda & 7) || (g.N & 1) ||
+      (reinterpret_cast<uintptr_t>(g.A) & 15) || (reinterpret_cast<uintptr_t>(g.W) & 15))
+    return launch_gemm_mma(g, epi, st);
+  switch (epi) {
+    case EPI_STORE: return launch_one<EPI_STORE>(g, status, st);
+    case EPI_RESIDUAL: return launch_one<EPI_RESIDUAL>(g, status, st);
+    case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(g, status, st);
+    case EPI_LMSTATS: return launch_one<EPI_LMSTATS>(g, status, st);
+  }
+  return D2C_EINVAL;
+}
+
 }  // namespace d2c

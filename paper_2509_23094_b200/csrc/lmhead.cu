@@ -48,7 +48,7 @@ int launch_lm_reduce(const float* st_max, const float* st_sum, const int32_t* st
   const int grid = ceil_div(max_rows, 4) < 148 * 4 ? ceil_div(max_rows, 4) : 148 * 4;
   lm_reduce_kernel<<<grid, 128, 0, st>>>(st_max, st_sum, st_arg, n_tiles, n_rows, lm_rows, sel_idx, row_seq,
                                          seq_len, conf, pred);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 

@@ -65,15 +65,15 @@ int launch_rollout(const RolloutArgs& a, cudaStream_t st) {
   const int L = a.seq_len;
   uint8_t* insel = reinterpret_cast<uint8_t*>(a.partial + (size_t)a.n_split * a.batch * L);
   rollout_init_kernel<<<dim3(ceil_div(L, 256), a.batch), 256, 0, st>>>(a, insel);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   const float* u = a.u0;
   float* bufs[2] = {a.u1, a.u0};
   for (int l = a.n_layers - 1; l >= 0; --l) {
     float* out = (l == 0) ? a.c : bufs[(a.n_layers - 1 - l) & 1];
     rollout_partial_kernel<<<dim3(ceil_div(L, 256), a.n_split, a.batch), 256, 0, st>>>(a, a.abar + (size_t)l * a.layer_stride, u);
-    D2C_CUDA_OK(cudaGetLastError());
+    D2C_LAUNCHED();
     rollout_combine_kernel<<<dim3(ceil_div(L, 256), a.batch), 256, 0, st>>>(a, insel, u, out);
-    D2C_CUDA_OK(cudaGetLastError());
+    D2C_LAUNCHED();
     u = out;
   }
   return D2C_OK;

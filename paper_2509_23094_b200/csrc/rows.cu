@@ -69,7 +69,7 @@ int launch_gather_norm(const bf16* h0, const int32_t* sel_idx, const int32_t* ro
   if (max_rows <= 0) return D2C_OK;
   norm_rows_kernel<true><<<row_grid(max_rows), kRowThreads, 0, st>>>(h0, sel_idx, row_seq, nullptr, n_rows,
                                                                       seq_len, d, gain, eps, x, xn);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 
@@ -78,7 +78,7 @@ int launch_rmsnorm(const bf16* x, const int32_t* row_map, const int32_t* n_rows,
   if (max_rows <= 0) return D2C_OK;
   norm_rows_kernel<false><<<row_grid(max_rows), kRowThreads, 0, st>>>(x, nullptr, nullptr, row_map, n_rows, 0, d,
                                                                        gain, eps, nullptr, xn);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 
@@ -96,7 +96,7 @@ __global__ void rope_table_kernel(float2* tab, int max_seq, int half, double bas
 int launch_rope_table(float2* tab, int max_seq, int head_dim, float base, cudaStream_t st) {
   const int half = head_dim / 2, n = max_seq * half;
   rope_table_kernel<<<ceil_div(n, 256), 256, 0, st>>>(tab, max_seq, half, (double)base, head_dim);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 
@@ -147,7 +147,7 @@ int launch_rope_scatter(bf16* qkv, const int32_t* sel_idx, const int32_t* row_se
   if (max_rows <= 0) return D2C_OK;
   rope_scatter_kernel<<<row_grid(max_rows), kRowThreads, 0, st>>>(qkv, sel_idx, row_seq, n_rows, hq, hkv, dh, rope,
                                                                    kc, vc, cache_seq);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 

@@ -246,10 +246,10 @@ int launch_select(const SelectArgs& a, cudaStream_t st) {
     attr_set = true;
   }
   select_kernel<<<a.batch, kSelThreads, smem, st>>>(a, P2);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   dim3 grid(ceil_div(a.seq_len, 256), a.batch);
   select_finalize_kernel<<<grid, 256, 0, st>>>(a);
-  D2C_CUDA_OK(cudaGetLastError());
+  D2C_LAUNCHED();
   return D2C_OK;
 }
 
