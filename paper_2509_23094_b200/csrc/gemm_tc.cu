@@ -2,16 +2,16 @@
 //
 //   C[m][n] = sum_k A[m][k] * W[n][k]      A: [max_rows][K] bf16, W: [N][K] bf16 (both K-major)
 //
-// One CTA computes one 128 x BN output tile (BN = 128, or 128 gate + 128 up columns for the SwiGLU
-// epilogue).  Warp roles:
+// Persistent CTAs (one per SM) walk over 128 x 256 accumulator tiles (256 output columns, or 128 gate +
+// 128 up columns for the SwiGLU epilogue).  Warp roles:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of 128 x 64 bf16 boxes (128-byte swizzle) into a
 //               ring of shared-memory stages, completion signalled on mbarriers;
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared-memory
-//               descriptors into a TMEM accumulator; tcgen05.commit releases each stage back to the
-//               producer and finally signals the epilogue;
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16) from shared-memory
+//               descriptors into one of two TMEM accumulators; tcgen05.commit releases each stage back
+//               to the producer and finally signals the epilogue;
 //   warps 2-5   epilogue: tcgen05.ld brings one accumulator row per thread into registers, the fused
 //               epilogue (bias / residual / SwiGLU / soft-max statistics) runs there, rows go to HBM.
-// The live row count is read from device memory: tiles past it exit before allocating anything.
+// The live row count is read from device memory: the tile list is derived from it on the device.
 // Every mbarrier wait is bounded; a wait that runs out raises D2C_ETIMEOUT in the status word, the
 // CTA drains its copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -111,45 +111,58 @@ union Pack8 { uint4 u; __nv_bfloat162 h[4]; };
 struct TcParams {
   GemmArgs g;
   int* status;
-  int stages;
 };
 
+constexpr int ST = 4;                            // shared-memory stages: 4 x (16 KB of A + 32 KB of B)
+constexpr int ACC_COLS = 256;                    // TMEM columns of one accumulator; two are allocated
+constexpr int B_BYTES = ACC_COLS * TK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...  Tiles are numbered with the row
+// tile fastest, so the CTAs that run together share one weight tile (read once from HBM, then L2).
+// A tile is 128 rows x 256 accumulator columns (for SwiGLU: 128 gate + 128 up columns of the same 128
+// outputs).  Two accumulators live in TMEM: the epilogue warps drain one while the MMA warp fills
+// the other.
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant__ CUtensorMap tmA64,
+               const __grid_constant__ CUtensorMap tmA32, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
-  constexpr int BN = (EPI == EPI_SWIGLU) ? 256 : 128;        // accumulator columns
-  constexpr int B_BYTES = BN * TK * 2;
-  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr int OUT_COLS = 128;                              // output columns per tile
+  constexpr int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : 256;  // output columns per tile
   const GemmArgs& g = p.g;
   const int n = *g.n_rows;
-  const int m0 = blockIdx.y * TM;
-  if (m0 >= n) return;                                       // uniform: nothing allocated yet
-  const int n0 = blockIdx.x * OUT_COLS;
+  if (n <= 0) return;
+  const int MT = (n + TM - 1) / TM, NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int total = MT * NT;
+  if ((int)blockIdx.x >= total) return;                      // uniform: nothing allocated yet
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int KT = g.K / TK, ST = p.stages;
+  const int KT = g.K / TK;
   int* status = p.status ? p.status : g_tc_status;
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
-  __shared__ __align__(8) uint64_t bars[2 * 8 + 1];          // full[ST], empty[ST], accumulator-ready
+  __shared__ __align__(8) uint64_t bars[2 * ST + 4];         // full[ST], empty[ST], acc_full[2], acc_empty[2]
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
-  const uint32_t acc_bar = bar0 + 8u * 16;
+  auto empty_bar = [&](int s) { return bar0 + 8u * (ST + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * ST + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * ST + 2 + b); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < ST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(acc_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), BN);
+    tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), 2 * ACC_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -161,23 +174,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued = 0;
-      for (int kt = 0; kt < KT; ++kt) {
-        const int s = kt % ST;
-        const uint32_t parity = ((kt / ST) & 1) ^ 1;          // a fresh barrier passes a wait on parity 1
-        if (!mbar_wait(empty_bar(s), parity, abortp, status, 1)) break;
-        const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-        mbar_expect_tx(full_bar(s), STAGE_BYTES);
-        tma_load_2d(sa, &tmA, kt * TK, m0, full_bar(s));
-        tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
-        if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
-        issued = kt + 1;
+      uint32_t it = 0;                                        // k-blocks issued so far (ring position)
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        const int m0 = (tile % MT) * TM, n0 = (tile / MT) * OUT_COLS;
+        const int rows = n - m0;                              // live rows of this tile: load no more than needed
+        const CUtensorMap* ma = rows <= 32 ? &tmA32 : (rows <= 64 ? &tmA64 : &tmA128);
+        const uint32_t a_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2;
+        for (int kt = 0; kt < KT; ++kt, ++it) {
+          const int s = it % ST;
+          if (!mbar_wait(empty_bar(s), ((it / ST) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx(full_bar(s), a_bytes + B_BYTES);
+          tma_load_2d(sa, ma, kt * TK, m0, full_bar(s));
+          tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
+          if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
+          else tma_load_2d(sb + 128 * TK * 2, &tmB, kt * TK, n0 + 128, full_bar(s));
+        }
       }
       if (*abortp) {
         // give the copies already in flight a bounded chance to land before the CTA goes away
-        for (int kt = max(0, issued - ST); kt < issued; ++kt) {
+        for (uint32_t j = it > (uint32_t)ST ? it - ST : 0; j < it; ++j) {
           const long long t0 = clock64();
-          while (!mbar_try_wait(full_bar(kt % ST), (kt / ST) & 1) && clock64() - t0 < kWaitCycles) {}
+          while (!mbar_try_wait(full_bar(j % ST), (j / ST) & 1) && clock64() - t0 < kWaitCycles) {}
         }
       }
     }
@@ -185,33 +204,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(BN);
+      constexpr uint32_t idesc = instr_desc(ACC_COLS);
+      uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int kt = 0; kt < KT && ok; ++kt) {
-        const int s = kt % ST;
-        ok = mbar_wait(full_bar(s), (kt / ST) & 1, abortp, status, 2);
-        if (!ok) break;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t buf = tcount & 1, use = tcount >> 1;
+        if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 4)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-        const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+        const uint32_t tacc = tmem_acc + buf * ACC_COLS;
+        for (int kt = 0; kt < KT; ++kt, ++it) {
+          const int s = it % ST;
+          if (!mbar_wait(full_bar(s), (it / ST) & 1, abortp, status, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
 #pragma unroll
-        for (int k = 0; k < TK / 16; ++k)                     // +32 bytes per K=16 slice inside the swizzle atom
-          umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
-        umma_commit(empty_bar(s));                            // stage reusable once these MMAs have read it
+          for (int k = 0; k < TK / 16; ++k)                   // +32 bytes per K=16 slice inside the swizzle atom
+            umma_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+          umma_commit(empty_bar(s));                          // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(acc_full(buf));                   // accumulator complete
       }
-      if (ok) umma_commit(acc_bar);                           // accumulator complete
     }
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;                             // TMEM lanes this warp may touch
     const int lrow = quarter * 32 + lane;
-    const int row = m0 + lrow;
-    const bool row_ok = row < n;
-    const bool ready = mbar_wait(acc_bar, 0, abortp, status, 3);
-    tc_fence_after();
-    if (ready) {
-      const uint32_t tbase = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tcount) {
+      const uint32_t buf = tcount & 1, use = tcount >> 1;
+      const int m0 = (tile % MT) * TM, nt = tile / MT, n0 = nt * OUT_COLS;
+      const int row = m0 + lrow;
+      const bool row_ok = row < n;
+      if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 3)) break;
+      tc_fence_after();
+      const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
@@ -285,40 +313,48 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
-        float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
 #pragma unroll 1
-        for (int c = 0; c < OUT_COLS / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tbase + c * 32, v);
-          tmem_ld_wait();
-          const int col0 = n0 + c * 32;
-          if (col0 >= g.N) continue;
-          float cmx = -INFINITY; int carg = 0x7fffffff;
+        for (int half = 0; half < 2; ++half) {                // statistics are kept per 128 columns
+          float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tbase + half * 128 + c * 32, v);
+            tmem_ld_wait();
+            const int col0 = n0 + half * 128 + c * 32;
+            if (col0 >= g.N) continue;
+            float cmx = -INFINITY; int carg = 0x7fffffff;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float f = __uint_as_float(v[j]);
-            if (col0 + j < g.N && f > cmx) { cmx = f; carg = col0 + j; }     // ascending columns: first maximum wins
-          }
-          const float nmx = fmaxf(mx, cmx);
-          float csum = 0.f;
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (col0 + j < g.N) csum += __expf(__uint_as_float(v[j]) - nmx);
-          sum = sum * __expf(mx - nmx) + csum;                                // exp(-inf) = 0 on the first chunk
-          if (cmx > mx) arg = carg;
-          mx = nmx;
-          if (g.logits && row_ok) {
-            float* lp = g.logits + (size_t)row * g.N + col0;
+            for (int j = 0; j < 32; ++j) {
+              const float f = __uint_as_float(v[j]);
+              if (col0 + j < g.N && f > cmx) { cmx = f; carg = col0 + j; }   // ascending columns: first maximum wins
+            }
+            const float nmx = fmaxf(mx, cmx);
+            float csum = 0.f;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              if (col0 + j < g.N) lp[j] = __uint_as_float(v[j]);
+              if (col0 + j < g.N) csum += __expf(__uint_as_float(v[j]) - nmx);
+            sum = sum * __expf(mx - nmx) + csum;                              // exp(-inf) = 0 on the first chunk
+            if (cmx > mx) arg = carg;
+            mx = nmx;
+            if (g.logits && row_ok) {
+              float* lp = g.logits + (size_t)row * g.N + col0;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < g.N) lp[j] = __uint_as_float(v[j]);
+            }
+          }
+          const int stile = nt * 2 + half;
+          if (row_ok && stile < g.n_tiles) {
+            const size_t o = (size_t)row * g.n_tiles + stile;
+            g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
           }
         }
-        if (row_ok) {
-          const size_t o = (size_t)row * g.n_tiles + blockIdx.x;
-          g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
-        }
       }
+      // hand the accumulator back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
     }
   }
   // ------------------------------------------------------------------ teardown
@@ -326,7 +362,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_acc, BN);
+    tmem_dealloc(tmem_acc, 2 * ACC_COLS);
   }
 }
 
@@ -346,14 +382,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D map over a row-major bf16 matrix [rows][cols] with leading dimension ld; box = 128 rows x 64 columns,
+// 2-D map over a row-major bf16 matrix [rows][cols] with leading dimension ld; box = box_rows x 64 columns,
 // 128-byte swizzle, out-of-range elements read as zero.
-int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) { set_global_error("cuTensorMapEncodeTiled is not available from this driver"); return D2C_ECUDA; }
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {ld * 2};
-  const cuuint32_t box[2] = {TK, TM};
+  const cuuint32_t box[2] = {TK, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -362,27 +398,36 @@ int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uin
   return D2C_OK;
 }
 
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
 template <int EPI>
 int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
-  constexpr int BN = (EPI == EPI_SWIGLU) ? 256 : 128;
-  constexpr int STAGE_BYTES = A_BYTES + BN * TK * 2;
-  const int stages = (EPI == EPI_SWIGLU) ? 4 : 6;
-  const int smem = stages * STAGE_BYTES + 1024;
+  const int smem = ST * STAGE_BYTES + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_set = true;
   }
-  CUtensorMap tmA, tmB, tmB2;
-  int rc = make_map(&tmA, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda);
+  CUtensorMap tmA128, tmA64, tmA32, tmB, tmB2;
+  int rc = make_map(&tmA128, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
+  if (rc == D2C_OK) rc = make_map(&tmA64, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 64);
+  if (rc == D2C_OK) rc = make_map(&tmA32, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 32);
+  if (rc == D2C_OK) rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
+  if (rc == D2C_OK) rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
   if (rc != D2C_OK) return rc;
-  rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K);
-  if (rc != D2C_OK) return rc;
-  rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K);
-  if (rc != D2C_OK) return rc;
-  TcParams p{g, status, stages};
-  dim3 grid(ceil_div(g.N, 128), ceil_div(g.max_rows, TM));
-  gemm_tc_kernel<EPI><<<grid, TC_THREADS, smem, st>>>(tmA, tmB, tmB2, p);
+  TcParams p{g, status};
+  const int out_cols = EPI == EPI_SWIGLU ? 128 : 256;
+  const long long tiles = (long long)ceil_div(g.max_rows, TM) * ceil_div(g.N, out_cols);
+  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  gemm_tc_kernel<EPI><<<grid, TC_THREADS, smem, st>>>(tmA128, tmA64, tmA32, tmB, tmB2, p);
   D2C_LAUNCHED();
   return D2C_OK;
 }
