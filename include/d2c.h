@@ -247,6 +247,22 @@ int d2c_op_rollout(const float* abar, size_t layer_stride, int32_t n_layers, con
                    const int32_t* row_off, int32_t batch, int32_t seq_len, float* c,
                    void* scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* d2c_op_rollout without a scratch argument.  (The paper has no counterpart for this entry point; it
+ * exists for integration reasons only.)  It serves callers that cannot get device memory at the time
+ * of the call, e.g. an inference server whose start-up handed every free byte of HBM to its cache
+ * arena, or code on a latency-critical stream that may not go through cudaMalloc and its implicit
+ * device synchronisation.  The scratch is a fixed array inside the library image (about 1.2 MB on every
+ * GPU that loads the library, until the process exits), which limits the call to
+ * batch * seq_len <= 16384; larger problems get D2C_ECAPACITY and should use d2c_op_rollout.
+ * Arguments, outputs and results are those of d2c_op_rollout.  Calls no cudaMalloc / cudaFree and no
+ * allocating library routine.  The first call on each device looks up the array's device address
+ * (with that device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array: two calls whose kernels may overlap on the GPU (different streams, no ordering
+ * between them) race on it, so order them.  Nothing in the array has to be cleared between calls:
+ * every word that is read has been written earlier in the same call. */
+int d2c_op_rollout_static(const float* abar, size_t layer_stride, int32_t n_layers, const int32_t* sel_idx,
+                          const int32_t* row_off, int32_t batch, int32_t seq_len, float* c, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ D2C_OK, D2C_EINVAL, D2C_ESHAPE, D2C_ECAPACITY, D2C_ECUDA, D2C_ETIMEOUT = 0, -1, 
 SYMBOLS = ["d2c_workspace_bytes", "d2c_create", "d2c_step", "d2c_step_host", "d2c_commit", "d2c_state_ptrs",
            "d2c_sync_status", "d2c_last_error", "d2c_destroy", "d2c_profile", "d2c_profile_read", "d2c_phase_name", "d2c_op_select_scratch_bytes", "d2c_op_select",
            "d2c_op_gemm", "d2c_op_attention", "d2c_op_lm_head_scratch_bytes", "d2c_op_lm_head",
-           "d2c_op_rollout_scratch_bytes", "d2c_op_rollout"]
+           "d2c_op_rollout_scratch_bytes", "d2c_op_rollout", "d2c_op_rollout_static"]
 
 
 class D2cError(RuntimeError):
@@ -100,6 +100,7 @@ def load() -> C.CDLL:
     lib.d2c_op_rollout_scratch_bytes.restype = sz
     lib.d2c_op_rollout_scratch_bytes.argtypes = [i32, i32]
     lib.d2c_op_rollout.argtypes = [vp, sz, i32, vp, vp, i32, i32, vp, vp, sz, vp]
+    lib.d2c_op_rollout_static.argtypes = [vp, sz, i32, vp, vp, i32, i32, vp, vp]
     for name in SYMBOLS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:
@@ -338,4 +339,14 @@ def d2c_op_rollout(abar, sel_idx, row_off, batch, seq_len, c=None):
     scratch = _scratch(nb, dev)
     _check(lib.d2c_op_rollout(_ptr(abar), layer_stride, n_layers, _ptr(sel_idx), _ptr(row_off), batch, seq_len,
                               _ptr(c), scratch.data_ptr(), nb, _stream_ptr()))
+    return c
+
+
+def d2c_op_rollout_static(abar, sel_idx, row_off, batch, seq_len, c=None):
+    """d2c_op_rollout for callers that cannot allocate: the scratch is a fixed array inside the library
+    (batch * seq_len <= 16384).  This wrapper itself only creates the output tensor when none is given."""
+    if c is None:
+        c = torch.zeros(batch, seq_len, dtype=torch.float32, device=abar.device)
+    _check(load().d2c_op_rollout_static(_ptr(abar), abar.stride(0), abar.shape[0], _ptr(sel_idx), _ptr(row_off), batch,
+                                        seq_len, _ptr(c), _stream_ptr()))
     return c
