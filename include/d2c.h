@@ -115,6 +115,8 @@ typedef struct {
   void*    hidden_out;  /* optional bf16 [max_batch*max_seq][d]: residual stream of the selected rows
                            after the last layer (rows beyond row_off[batch] are not written)             */
   float*   logits;      /* optional f32 [rows with a masked position][V] in row order (debug, slow path)  */
+  void*    layer_in;    /* optional bf16 [n_layers][batch*seq_len][d]: the residual stream of the selected
+                           rows as it enters each layer (debug: lets a checker verify one layer at a time) */
 } d2c_step_out;
 
 /* One decoding step (see the top of this file).  Device pointers; enqueues only.

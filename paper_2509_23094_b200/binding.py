@@ -49,7 +49,8 @@ class StepArgs(C.Structure):
 
 
 class StepOut(C.Structure):
-    _fields_ = [("sel_idx", C.c_void_p), ("row_off", C.c_void_p), ("hidden_out", C.c_void_p), ("logits", C.c_void_p)]
+    _fields_ = [("sel_idx", C.c_void_p), ("row_off", C.c_void_p), ("hidden_out", C.c_void_p), ("logits", C.c_void_p),
+                ("layer_in", C.c_void_p)]
 
 
 class HostOut(C.Structure):
@@ -178,8 +179,8 @@ class Context:
 
     # -- views into the workspace (no copies) ------------------------------------------------
     def _view(self, ptr: int, numel: int, dtype: torch.dtype) -> torch.Tensor:
-        off = ptr - self.workspace.data_ptr()
-        nbytes = numel * torch.empty(0, dtype=dtype).element_size()
+        off = int(ptr) - self.workspace.data_ptr()
+        nbytes = int(numel) * torch.empty(0, dtype=dtype).element_size()
         return self.workspace[off: off + nbytes].view(dtype)
 
     def view(self, name: str, batch: Optional[int] = None, seq_len: Optional[int] = None) -> torch.Tensor:
@@ -207,8 +208,9 @@ class Context:
 
     def abar(self, layer: int, n_rows: int, seq_len: int) -> torch.Tensor:
         c = self.cfg
+        n_rows, seq_len = int(n_rows), int(seq_len)
         stride = c.max_batch * c.max_seq * c.max_seq
-        ptr = self.state.abar + layer * stride * 4
+        ptr = self.state.abar + int(layer) * stride * 4
         return self._view(ptr, n_rows * seq_len, torch.float32).view(n_rows, seq_len)
 
     # -- entry points ---------------------------------------------------------------------------
@@ -216,11 +218,11 @@ class Context:
              forced_off: Optional[torch.Tensor] = None, override_key: Optional[torch.Tensor] = None,
              override_c: Optional[torch.Tensor] = None, hidden_out: Optional[torch.Tensor] = None,
              sel_idx: Optional[torch.Tensor] = None, row_off: Optional[torch.Tensor] = None,
-             logits: Optional[torch.Tensor] = None) -> None:
+             logits: Optional[torch.Tensor] = None, layer_in: Optional[torch.Tensor] = None) -> None:
         B, L = mask.shape
         a = StepArgs(B, L, _ptr(h0), _ptr(mask), _ptr(forced), _ptr(forced_off), int(k), float(p),
                      _ptr(override_key), _ptr(override_c))
-        o = StepOut(_ptr(sel_idx), _ptr(row_off), _ptr(hidden_out), _ptr(logits))
+        o = StepOut(_ptr(sel_idx), _ptr(row_off), _ptr(hidden_out), _ptr(logits), _ptr(layer_in))
         _check(load().d2c_step(self.handle, C.byref(a), C.byref(o)), self.handle)
 
     def step_host(self, h0: torch.Tensor, mask: torch.Tensor, k: int, p: float, forced=None, forced_off=None,

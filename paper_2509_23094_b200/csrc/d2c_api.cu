@@ -276,6 +276,11 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   D2C_TRY(ctx, launch_gather_norm((const bf16*)a->h0, b.sel_idx, b.row_seq, n_rows, R, L, d, ctx->g_attn[0], c.rms_eps, x, b.xn, st));
   const int depth = rollout_depth(c);
   for (int l = 0; l < c.n_layers; ++l) {
+    if (out && out->layer_in) {
+      cudaError_t e = cudaMemcpyAsync(static_cast<bf16*>(out->layer_in) + (size_t)l * R * d, x, (size_t)R * d * sizeof(bf16),
+                                      cudaMemcpyDeviceToDevice, st);
+      if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
+    }
     if (l > 0) {
       D2C_TRY(ctx, mark(ctx, PH_NORM));
       D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
