@@ -67,7 +67,8 @@ typedef struct {
   int32_t rollout_layers;     /* 0: rollout over all layers (Eq. 8); n>0: only the first n layers        */
   int32_t flags;              /* D2C_FLAG_* bits                                                         */
 } d2c_config;
-#define D2C_FLAG_PORTABLE_GEMM 1   /* run the GEMMs on the mma.sync kernel instead of the tcgen05 one (cross-check) */
+#define D2C_FLAG_PORTABLE_GEMM 1        /* run the GEMMs on the mma.sync kernel instead of the tcgen05 one (cross-check) */
+#define D2C_FLAG_PORTABLE_ATTENTION 2   /* same for the attention kernels                                                */
 
 /* Weights.  The arrays of per-layer pointers are HOST arrays of n_layers DEVICE
  * pointers; they are copied at create, the device memory is borrowed for the
@@ -218,15 +219,16 @@ int d2c_op_gemm(const void* A, const void* W, const void* bias, void* C, const i
                 int32_t max_rows, int32_t N, int32_t K, int32_t impl, void* cuda_stream);
 
 /* Selected-query bidirectional attention of one layer (Section 4.2).
- * q: bf16 [rows][ldq] with head h at columns [h*Dh,(h+1)*Dh) (already rotated);
+ * q: bf16 [q_rows][ldq] with head h at columns [h*Dh,(h+1)*Dh) (already rotated); q_rows >= row_off[batch];
  * kcache/vcache: bf16 [batch][cache_seq][Hkv][Dh] of this layer; rows of sequence b are
  * [row_off[b], row_off[b+1]) and attend to keys 0..seq_len-1 of that sequence.
  * Outputs: o bf16 [rows][Hq*Dh]; lse f32 [rows][Hq] (natural log); abar f32
- * [rows][seq_len] = mean over the Hq heads of the softmax probabilities. */
-int d2c_op_attention(const void* q, int32_t ldq, const void* kcache, const void* vcache,
+ * [rows][seq_len] = mean over the Hq heads of the softmax probabilities (may be NULL).
+ * impl 0: tcgen05 kernels where the shape allows (head_dim 128, q_rows >= 128), impl 1: mma.sync kernels. */
+int d2c_op_attention(const void* q, int32_t q_rows, int32_t ldq, const void* kcache, const void* vcache,
                      const int32_t* row_off, int32_t batch, int32_t seq_len, int32_t cache_seq,
                      int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
-                     void* o, float* lse, float* abar, void* cuda_stream);
+                     void* o, float* lse, float* abar, int32_t impl, void* cuda_stream);
 
 /* Bytes of scratch d2c_op_lm_head needs for up to max_rows rows. */
 size_t d2c_op_lm_head_scratch_bytes(int32_t max_rows, int32_t vocab);

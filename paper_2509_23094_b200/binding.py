@@ -94,7 +94,7 @@ def load() -> C.CDLL:
     lib.d2c_op_select_scratch_bytes.argtypes = [i32, i32]
     lib.d2c_op_select.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.d2c_op_gemm.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
-    lib.d2c_op_attention.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.d2c_op_attention.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.d2c_op_lm_head_scratch_bytes.restype = sz
     lib.d2c_op_lm_head_scratch_bytes.argtypes = [i32, i32]
     lib.d2c_op_lm_head.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -303,15 +303,15 @@ def d2c_op_gemm(A, W, n_rows, bias=None, impl=0):
     return Cm
 
 
-def d2c_op_attention(q, kcache, vcache, row_off, seq_len, n_q_heads, n_kv_heads, head_dim, want_abar=True):
+def d2c_op_attention(q, kcache, vcache, row_off, seq_len, n_q_heads, n_kv_heads, head_dim, want_abar=True, impl=0):
     rows, ldq = q.shape
     B, cache_seq = kcache.shape[0], kcache.shape[1]
     dev = q.device
     o = torch.zeros(rows, n_q_heads * head_dim, dtype=torch.bfloat16, device=dev)
     lse = torch.zeros(rows, n_q_heads, dtype=torch.float32, device=dev)
     abar = torch.zeros(rows, seq_len, dtype=torch.float32, device=dev) if want_abar else None
-    _check(load().d2c_op_attention(_ptr(q), ldq, _ptr(kcache), _ptr(vcache), _ptr(row_off), B, seq_len, cache_seq,
-                                   n_q_heads, n_kv_heads, head_dim, _ptr(o), _ptr(lse), _ptr(abar), _stream_ptr()))
+    _check(load().d2c_op_attention(_ptr(q), rows, ldq, _ptr(kcache), _ptr(vcache), _ptr(row_off), B, seq_len, cache_seq,
+                                   n_q_heads, n_kv_heads, head_dim, _ptr(o), _ptr(lse), _ptr(abar), int(impl), _stream_ptr()))
     return o, lse, abar
 
 

@@ -268,6 +268,7 @@ int launch_dh(const AttnArgs& a, cudaStream_t st) {
 int launch_attention(const AttnArgs& a, cudaStream_t st) {
   if (a.batch <= 0 || a.seq_len <= 0 || a.max_rows_per_seq <= 0) return D2C_OK;
   if (a.hq % a.hkv != 0) { set_global_error("attention: %d query heads not a multiple of %d kv heads", a.hq, a.hkv); return D2C_ESHAPE; }
+  if (!a.portable && attention_tc_supported(a)) return launch_attention_tc(a, st, a.status);
   if (a.dh == 64) return launch_dh<64>(a, st);
   if (a.dh == 128) return launch_dh<128>(a, st);
   set_global_error("attention: head_dim %d not supported (64 or 128)", a.dh);

@@ -1,0 +1,504 @@
+// Selected-query bidirectional attention on the 5th-generation tensor cores (head_dim 128).
+//
+//   attn_fwd_tc    O = softmax(Q K^T / sqrt(Dh)) V and the log-sum-exp per (row, head).  One CTA per
+//                  (128 selected rows, head, sequence); keys stream in tiles of 128 through TMA.
+//                  S = Q K^T is a tcgen05.mma into TMEM; four softmax warps (one row per thread) read it
+//                  with tcgen05.ld, write the bf16 probabilities back over the same TMEM columns and the
+//                  PV product takes them from there as its A operand (V is the MN-major B operand straight
+//                  from the TMA tile).  Each tile's PV lands in its own TMEM buffer and is folded into
+//                  fp32 registers with the usual running-max rescale, so no TMEM read-modify-write exists.
+//   attn_abar_tc   Abar[r][j] = 1/Hq sum_h exp(s_h[r][j] - lse_h[r]) (Section 4.2): one CTA per
+//                  (128 rows x 128 keys) loops over the heads, S by tcgen05.mma, the sum over heads in
+//                  registers in a fixed order (deterministic).
+//
+// Warp roles in both: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-5 softmax/epilogue.
+// No cluster, no multicast.  Every mbarrier wait is bounded (see gemm_tc.cu for the protocol).
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace d2c {
+namespace {
+
+constexpr int AQ = 128, AKEYS = 128, ADH = 128;
+constexpr int HALF_BYTES = 128 * 64 * 2;          // one 128-row x 64-column swizzled box: 16 KB
+constexpr int TILE_BYTES = 2 * HALF_BYTES;        // 128 x 128 bf16
+constexpr int ATC_THREADS = 192;
+constexpr long long kWaitCycles = 4000000000LL;
+constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+
+__device__ int g_attn_status[4];
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile("{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
+               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = site;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                 "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                 "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                 "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+               ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                 "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// K-major bf16 tile of 128-byte swizzled rows (8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+// MN-major bf16 operand: 64 contiguous N elements per 128-byte row, 8 K-rows per 1024-byte group
+// (stride offset), the next 64 N elements 16 KB further (leading offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(HALF_BYTES >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// bf16 x bf16 -> fp32, M = 128, N = 128; bit 16 set: B is MN-major.
+constexpr uint32_t kIdescKK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescKMn = kIdescKK | (1u << 16);
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+struct AttnTcParams { AttnArgs a; int* status; };
+
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ATC_THREADS, 1)
+attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+            const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+  const AttnArgs& a = p.a;
+  const int b = blockIdx.z, h = blockIdx.y, g = h / (a.hq / a.hkv);
+  const int r0 = a.row_off[b] + blockIdx.x * AQ;
+  const int nrows = min(AQ, a.row_off[b + 1] - r0);
+  if (nrows <= 0) return;                                          // uniform: nothing allocated yet
+  const int L = a.seq_len, T = (L + AKEYS - 1) / AKEYS;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int* status = p.status ? p.status : g_attn_status;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t sQ = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
+  auto sK = [&](int s) { return sQ + TILE_BYTES + s * 2 * TILE_BYTES; };
+  auto sV = [&](int s) { return sK(s) + TILE_BYTES; };
+  // barriers: 0 q_full | 1,2 k_full | 3,4 v_full | 5,6 kv_empty | 7,8 s_full | 9,10 p_full | 11,12 o_full | 13,14 o_empty
+  __shared__ __align__(8) uint64_t bars[15];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  auto B = [&](int i) { return bar0 + 8u * i; };
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 9; ++i) mbar_init(B(i), 1);
+    mbar_init(B(9), 4); mbar_init(B(10), 4);
+    mbar_init(B(11), 1); mbar_init(B(12), 1);
+    mbar_init(B(13), 4); mbar_init(B(14), 4);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) { tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tm = tmem_slot;                                    // S/P buffers at +0, +128; PV buffers at +256, +384
+  volatile int* abortp = &abort_flag;
+  const int kv_row0 = b * a.cache_seq;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(B(0), TILE_BYTES);
+      tma_load_2d(sQ, &tmQ, h * ADH, r0, B(0));
+      tma_load_2d(sQ + HALF_BYTES, &tmQ, h * ADH + 64, r0, B(0));
+      int issued = 0;
+      for (int j = 0; j < T; ++j) {
+        const int s = j & 1, u = j >> 1;
+        if (!mbar_wait(B(5 + s), (u & 1) ^ 1, abortp, status, 11)) break;
+        mbar_expect_tx(B(1 + s), TILE_BYTES);
+        tma_load_2d(sK(s), &tmK, g * ADH, kv_row0 + j * AKEYS, B(1 + s));
+        tma_load_2d(sK(s) + HALF_BYTES, &tmK, g * ADH + 64, kv_row0 + j * AKEYS, B(1 + s));
+        mbar_expect_tx(B(3 + s), TILE_BYTES);
+        tma_load_2d(sV(s), &tmV, g * ADH, kv_row0 + j * AKEYS, B(3 + s));
+        tma_load_2d(sV(s) + HALF_BYTES, &tmV, g * ADH + 64, kv_row0 + j * AKEYS, B(3 + s));
+        issued = j + 1;
+      }
+      if (*abortp) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(B(0), 0) && clock64() - t0 < kWaitCycles) {}
+        for (int j = max(0, issued - 2); j < issued; ++j) {
+          const long long t1 = clock64();
+          while (!(mbar_try_wait(B(1 + (j & 1)), (j >> 1) & 1) && mbar_try_wait(B(3 + (j & 1)), (j >> 1) & 1)) &&
+                 clock64() - t1 < kWaitCycles) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = mbar_wait(B(0), 0, abortp, status, 12);
+      auto issue_s = [&](int j) {                                   // S_j = Q K_j^T into buffer j & 1
+        const int s = j & 1;
+        if (!mbar_wait(B(1 + s), (j >> 1) & 1, abortp, status, 13)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int i = 0; i < ADH / 16; ++i) {
+          const uint32_t off = (i >> 2) * HALF_BYTES;
+          umma_ss(tm + s * 128, desc_kmajor(sQ + off) + 2 * (i & 3), desc_kmajor(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
+        }
+        umma_commit(B(7 + s));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < T && ok; ++j) {
+        const int s = j & 1, u = j >> 1;
+        if (j + 1 < T) { ok = issue_s(j + 1); if (!ok) break; }
+        if (!mbar_wait(B(9 + s), u & 1, abortp, status, 14) || !mbar_wait(B(3 + s), u & 1, abortp, status, 15) ||
+            !mbar_wait(B(13 + s), (u & 1) ^ 1, abortp, status, 16)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int i = 0; i < AKEYS / 16; ++i)                       // P_j (TMEM, 8 columns per 16 keys) x V_j
+          umma_ts(tm + 256 + s * 128, tm + s * 128 + 8 * i, desc_mnmajor(sV(s) + i * 2048), kIdescKMn, i != 0);
+        umma_commit(B(5 + s));                                      // K/V stage free
+        umma_commit(B(11 + s));                                     // PV_j ready
+      }
+    }
+    __syncwarp();
+  } else {
+    const int quarter = warp & 3, lrow = quarter * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const float sc = kLog2e * rsqrtf((float)ADH);
+    float o[ADH];
+#pragma unroll
+    for (int i = 0; i < ADH; ++i) o[i] = 0.f;
+    float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
+    bool ok = true;
+    auto fold_pv = [&](int j, float alpha) {                        // o = o * alpha + PV_j
+      const int s = j & 1;
+      if (!mbar_wait(B(11 + s), (j >> 1) & 1, abortp, status, 17)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tm + 256 + s * 128 + lane_base + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(v[i]));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(13 + s));
+      return true;
+    };
+    for (int j = 0; j < T && ok; ++j) {
+      const int s = j & 1;
+      if (!mbar_wait(B(7 + s), (j >> 1) & 1, abortp, status, 18)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t ts = tm + s * 128 + lane_base;
+      const int key0 = j * AKEYS;
+      float mx = m;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {                                 // pass 1: running maximum
+        uint32_t v[32];
+        tmem_ld32(ts + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (key0 + c * 32 + i < L) mx = fmaxf(mx, __uint_as_float(v[i]) * sc);
+      }
+      const float alpha = exp2f(m - mx);                            // first tile: exp2(-inf) = 0
+      m = mx;
+      float rs = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {                                 // pass 2: probabilities, written back as bf16
+        uint32_t v[32], pk[16];
+        tmem_ld32(ts + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int k = key0 + c * 32 + 2 * i;
+          const float p0 = k < L ? exp2f(__uint_as_float(v[2 * i]) * sc - m) : 0.f;
+          const float p1 = k + 1 < L ? exp2f(__uint_as_float(v[2 * i + 1]) * sc - m) : 0.f;
+          rs += p0 + p1;
+          pk[i] = pack_bf16(p0, p1);
+        }
+        tmem_st16(ts + c * 16, pk);                                 // lands on columns whose scores are already consumed
+      }
+      l = l * alpha + rs;
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(9 + s));
+      if (j >= 1) ok = fold_pv(j - 1, alpha_prev);
+      alpha_prev = alpha;
+    }
+    if (ok) ok = fold_pv(T - 1, alpha_prev);
+    if (ok && lrow < nrows) {
+      const float inv = 1.f / l;
+      bf16* dst = a.o + (size_t)(r0 + lrow) * ((size_t)a.hq * ADH) + (size_t)h * ADH;
+#pragma unroll
+      for (int q = 0; q < ADH / 8; ++q) {
+        uint4 w;
+        w.x = pack_bf16(o[q * 8 + 0] * inv, o[q * 8 + 1] * inv); w.y = pack_bf16(o[q * 8 + 2] * inv, o[q * 8 + 3] * inv);
+        w.z = pack_bf16(o[q * 8 + 4] * inv, o[q * 8 + 5] * inv); w.w = pack_bf16(o[q * 8 + 6] * inv, o[q * 8 + 7] * inv);
+        reinterpret_cast<uint4*>(dst)[q] = w;
+      }
+      a.lse[(size_t)(r0 + lrow) * a.hq + h] = (m + log2f(l)) * kLn2;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tm, 512); }
+}
+
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ATC_THREADS, 1)
+attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const AttnTcParams p) {
+  const AttnArgs& a = p.a;
+  const int b = blockIdx.z;
+  const int r0 = a.row_off[b] + blockIdx.y * AQ;
+  const int nrows = min(AQ, a.row_off[b + 1] - r0);
+  const int key0 = blockIdx.x * AKEYS, L = a.seq_len;
+  if (nrows <= 0 || key0 >= L) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = a.hq / a.hkv;
+  int* status = p.status ? p.status : g_attn_status;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
+  auto sQ = [&](int s) { return base + s * TILE_BYTES; };           // two Q stages, then two K stages
+  auto sK = [&](int s) { return base + (2 + s) * TILE_BYTES; };
+  // barriers: 0,1 q_full | 2,3 k_full | 4,5 q_empty | 6,7 k_empty | 8,9 s_full | 10,11 s_empty
+  __shared__ __align__(8) uint64_t bars[12];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  auto B = [&](int i) { return bar0 + 8u * i; };
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 10; ++i) mbar_init(B(i), 1);
+    mbar_init(B(10), 4); mbar_init(B(11), 4);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) { tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), 256); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tm = tmem_slot;
+  volatile int* abortp = &abort_flag;
+  const int kv_row = b * a.cache_seq + key0;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = 0;
+      for (int h = 0; h < a.hq; ++h) {
+        const int s = h & 1, u = h >> 1;
+        if (!mbar_wait(B(4 + s), (u & 1) ^ 1, abortp, status, 21)) break;
+        mbar_expect_tx(B(s), TILE_BYTES);
+        tma_load_2d(sQ(s), &tmQ, h * ADH, r0, B(s));
+        tma_load_2d(sQ(s) + HALF_BYTES, &tmQ, h * ADH + 64, r0, B(s));
+        if (h % group == 0) {
+          const int gi = h / group, ks = gi & 1, ku = gi >> 1;
+          if (!mbar_wait(B(6 + ks), (ku & 1) ^ 1, abortp, status, 22)) break;
+          mbar_expect_tx(B(2 + ks), TILE_BYTES);
+          tma_load_2d(sK(ks), &tmK, gi * ADH, kv_row, B(2 + ks));
+          tma_load_2d(sK(ks) + HALF_BYTES, &tmK, gi * ADH + 64, kv_row, B(2 + ks));
+        }
+        issued = h + 1;
+      }
+      if (*abortp) {
+        for (int h = max(0, issued - 2); h < issued; ++h) {
+          const long long t1 = clock64();
+          while (!mbar_try_wait(B(h & 1), (h >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      for (int h = 0; h < a.hq; ++h) {
+        const int s = h & 1, u = h >> 1, gi = h / group, ks = gi & 1, ku = gi >> 1;
+        if (!mbar_wait(B(s), u & 1, abortp, status, 23)) break;
+        if (h % group == 0 && !mbar_wait(B(2 + ks), ku & 1, abortp, status, 24)) break;
+        if (!mbar_wait(B(10 + s), (u & 1) ^ 1, abortp, status, 25)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int i = 0; i < ADH / 16; ++i) {
+          const uint32_t off = (i >> 2) * HALF_BYTES;
+          umma_ss(tm + s * 128, desc_kmajor(sQ(s) + off) + 2 * (i & 3), desc_kmajor(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
+        }
+        umma_commit(B(4 + s));                                      // Q stage free
+        if ((h + 1) % group == 0 || h + 1 == a.hq) umma_commit(B(6 + ks));   // last head of the group: K stage free
+        umma_commit(B(8 + s));
+      }
+    }
+    __syncwarp();
+  } else {
+    const int quarter = warp & 3, lrow = quarter * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const float sc = kLog2e * rsqrtf((float)ADH);
+    const bool row_ok = lrow < nrows;
+    float acc[AKEYS];
+#pragma unroll
+    for (int i = 0; i < AKEYS; ++i) acc[i] = 0.f;
+    bool ok = true;
+    for (int h = 0; h < a.hq && ok; ++h) {
+      const int s = h & 1;
+      const float e = row_ok ? a.lse[(size_t)(r0 + lrow) * a.hq + h] * kLog2e : 0.f;
+      if (!mbar_wait(B(8 + s), (h >> 1) & 1, abortp, status, 26)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tm + s * 128 + lane_base + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[c * 32 + i] += exp2f(__uint_as_float(v[i]) * sc - e);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(B(10 + s));
+    }
+    if (ok && row_ok) {
+      const float inv = 1.f / (float)a.hq;
+      float* dst = a.abar + (size_t)(r0 + lrow) * L + key0;
+      if (key0 + AKEYS <= L && (L & 3) == 0) {
+#pragma unroll
+        for (int q = 0; q < AKEYS / 4; ++q)
+          reinterpret_cast<float4*>(dst)[q] = make_float4(acc[4 * q] * inv, acc[4 * q + 1] * inv, acc[4 * q + 2] * inv, acc[4 * q + 3] * inv);
+      } else {
+#pragma unroll
+        for (int i = 0; i < AKEYS; ++i)
+          if (key0 + i < L) dst[i] = acc[i] * inv;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tm, 256); }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+// [rows][cols] bf16, leading dimension ld, box 128 rows x 64 columns, 128-byte swizzle, zero fill.
+int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_global_error("cuTensorMapEncodeTiled is not available from this driver"); return D2C_ECUDA; }
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_global_error("cuTensorMapEncodeTiled failed with code %d", (int)r); return D2C_ECUDA; }
+  return D2C_OK;
+}
+}  // namespace
+
+// True if the tcgen05 kernels can take this problem (otherwise the caller uses the mma.sync ones).
+bool attention_tc_supported(const AttnArgs& a) {
+  return a.dh == ADH && a.q_rows >= AQ && (long long)a.batch * a.cache_seq >= AKEYS && (a.ldq & 7) == 0 &&
+         (reinterpret_cast<uintptr_t>(a.q) & 15) == 0 && (reinterpret_cast<uintptr_t>(a.kc) & 15) == 0 &&
+         (reinterpret_cast<uintptr_t>(a.vc) & 15) == 0;
+}
+
+int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
+  const int smem_fwd = 5 * TILE_BYTES + 1024, smem_ab = 4 * TILE_BYTES + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    D2C_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_fwd));
+    D2C_CUDA_OK(cudaFuncSetAttribute(attn_abar_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_ab));
+    attr_set = true;
+  }
+  CUtensorMap tmQ, tmK, tmV;
+  const uint64_t kv_cols = (uint64_t)a.hkv * a.dh, kv_rows = (uint64_t)a.batch * a.cache_seq;
+  int rc = make_map(&tmQ, a.q, (uint64_t)a.q_rows, (uint64_t)a.hq * a.dh, (uint64_t)a.ldq);
+  if (rc == D2C_OK) rc = make_map(&tmK, a.kc, kv_rows, kv_cols, kv_cols);
+  if (rc == D2C_OK) rc = make_map(&tmV, a.vc, kv_rows, kv_cols, kv_cols);
+  if (rc != D2C_OK) return rc;
+  AttnTcParams p{a, status};
+  const int qtiles = ceil_div(a.max_rows_per_seq, AQ);
+  attn_fwd_tc<<<dim3(qtiles, a.hq, a.batch), ATC_THREADS, smem_fwd, st>>>(tmQ, tmK, tmV, p);
+  D2C_LAUNCHED();
+  if (a.abar) {
+    attn_abar_tc<<<dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), ATC_THREADS, smem_ab, st>>>(tmQ, tmK, p);
+    D2C_LAUNCHED();
+  }
+  return D2C_OK;
+}
+
+}  // namespace d2c

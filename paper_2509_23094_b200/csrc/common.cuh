@@ -77,8 +77,13 @@ struct AttnArgs {
   const bf16* q; int ldq; const bf16* kc; const bf16* vc; const int32_t* row_off;
   int batch, seq_len, cache_seq, hq, hkv, dh; int max_rows_per_seq;
   bf16* o; float* lse; float* abar;      // abar may be null (layers outside the rollout)
+  int q_rows;                            // rows the q buffer holds (bounds the TMA map)
+  int portable;                          // 1: force the mma.sync kernels
+  int* status;                           // device status word for bounded waits (may be null)
 };
 int launch_attention(const AttnArgs& a, cudaStream_t st);
+bool attention_tc_supported(const AttnArgs& a);               // attention_tc.cu
+int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status);
 
 // ---- LM head statistics (lmhead.cu) ------------------------------------------------------------
 int launch_lm_reduce(const float* st_max, const float* st_sum, const int32_t* st_arg, int n_tiles,

@@ -92,7 +92,7 @@ static const char* check_config(const d2c_config* c) {
   if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
   if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
   if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
-  if (c->rollout_layers < 0 || (c->flags & ~D2C_FLAG_PORTABLE_GEMM)) return "rollout_layers >= 0 and no unknown flag bits required";
+  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION))) return "rollout_layers >= 0 and no unknown flag bits required";
   return nullptr;
 }
 
@@ -296,6 +296,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     AttnArgs at{};
     at.q = b.qkv; at.ldq = qkv_out; at.kc = kc; at.vc = vc; at.row_off = b.row_off; at.batch = B; at.seq_len = L;
     at.cache_seq = c.max_seq; at.hq = hq; at.hkv = hkv; at.dh = dh; at.max_rows_per_seq = L;
+    at.q_rows = R; at.portable = (c.flags & D2C_FLAG_PORTABLE_ATTENTION) ? 1 : 0; at.status = b.status;
     at.o = b.o; at.lse = b.lse; at.abar = l < depth ? b.abar + (size_t)l * c.max_batch * c.max_seq * c.max_seq : nullptr;
     D2C_TRY(ctx, mark(ctx, PH_ATTN));
     D2C_TRY(ctx, launch_attention(at, st));

@@ -66,17 +66,19 @@ int d2c_op_gemm(const void* A, const void* W, const void* bias, void* C, const i
   return bad(D2C_EINVAL, "d2c_op_gemm: impl must be 0 (tcgen05) or 1 (mma.sync)");
 }
 
-int d2c_op_attention(const void* q, int32_t ldq, const void* kcache, const void* vcache,
+int d2c_op_attention(const void* q, int32_t q_rows, int32_t ldq, const void* kcache, const void* vcache,
                      const int32_t* row_off, int32_t batch, int32_t seq_len, int32_t cache_seq,
                      int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
-                     void* o, float* lse, float* abar, void* cuda_stream) {
+                     void* o, float* lse, float* abar, int32_t impl, void* cuda_stream) {
   if (!q || !kcache || !vcache || !row_off || !o || !lse) return bad(D2C_EINVAL, "d2c_op_attention: null pointer");
-  if (batch < 1 || seq_len < 1 || cache_seq < seq_len || n_q_heads < 1 || n_kv_heads < 1 || ldq < n_q_heads * head_dim || (ldq & 7))
+  if (batch < 1 || seq_len < 1 || cache_seq < seq_len || n_q_heads < 1 || n_kv_heads < 1 || ldq < n_q_heads * head_dim || (ldq & 7) ||
+      q_rows < 1 || (impl != 0 && impl != 1))
     return bad(D2C_EINVAL, "d2c_op_attention: bad sizes");
   AttnArgs a{};
   a.q = (const bf16*)q; a.ldq = ldq; a.kc = (const bf16*)kcache; a.vc = (const bf16*)vcache; a.row_off = row_off;
   a.batch = batch; a.seq_len = seq_len; a.cache_seq = cache_seq; a.hq = n_q_heads; a.hkv = n_kv_heads; a.dh = head_dim;
-  a.max_rows_per_seq = seq_len; a.o = (bf16*)o; a.lse = lse; a.abar = abar;
+  a.max_rows_per_seq = seq_len < q_rows ? seq_len : q_rows; a.o = (bf16*)o; a.lse = lse; a.abar = abar;
+  a.q_rows = q_rows; a.portable = impl; a.status = nullptr;
   return launch_attention(a, static_cast<cudaStream_t>(cuda_stream));
 }
 

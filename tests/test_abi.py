@@ -39,7 +39,7 @@ def test_workspace_bytes_and_config_validation(lib):
     big = binding.d2c_workspace_bytes(binding.make_config(inputs.LLADA_8B, 8, 4096))
     assert big > 2 * 32 * 8 * 4096 * 4096 * 2
     for field, val in [("head_dim", 96), ("d_model", 100), ("n_kv_heads", 3), ("max_seq", 10000), ("vocab", 1001),
-                       ("sigma", 0.0), ("flags", 2), ("stage2_candidates", 2)]:
+                       ("sigma", 0.0), ("flags", 4), ("stage2_candidates", 2)]:
         bad = binding.make_config(inputs.TOY, 1, 128)
         setattr(bad, field, val)
         assert binding.d2c_workspace_bytes(bad) == 0, field
@@ -72,6 +72,6 @@ def test_ops_reject_bad_arguments_without_a_device(lib):
     assert lib.d2c_op_gemm(256, 256, None, 256, 256, 8, 8, 32, 1, None) == binding.D2C_EINVAL
     assert lib.d2c_op_select(None, None, None, None, None, None, 1, 1, 0, 0.5, 10.0, 0, None, None, None, None, None,
                              None, None, 0, None) == binding.D2C_EINVAL
-    assert lib.d2c_op_attention(None, 0, None, None, None, 1, 1, 1, 1, 1, 64, None, None, None, None) == binding.D2C_EINVAL
+    assert lib.d2c_op_attention(None, 1, 0, None, None, None, 1, 1, 1, 1, 1, 64, None, None, None, 0, None) == binding.D2C_EINVAL
     assert lib.d2c_op_lm_head(None, None, None, 1, 64, 2, None, None, None, None, 0, None) == binding.D2C_EINVAL
     assert lib.d2c_op_rollout(None, 0, 1, None, None, 1, 1, None, None, 0, None) == binding.D2C_EINVAL

@@ -48,17 +48,20 @@ def _attention_ref(q, kc, vc, row_off, L, Hq, Hkv, Dh):
     return o, lse, abar
 
 
+@pytest.mark.parametrize("impl", [0, 1])
 @pytest.mark.parametrize("Hq,Hkv,Dh,L,cache_seq,nbs", [(4, 4, 64, 128, 128, [95]), (4, 2, 64, 200, 256, [1, 130]),
                                                          (4, 1, 128, 333, 400, [64, 0, 65]), (8, 8, 128, 64, 64, [64]),
-                                                         (2, 2, 128, 1000, 1024, [129])])
-def test_attention_matches_fp64(Hq, Hkv, Dh, L, cache_seq, nbs):
+                                                         (2, 2, 128, 1000, 1024, [129]), (4, 2, 128, 128, 128, [128, 128]),
+                                                         (6, 2, 128, 700, 768, [300, 5, 257])])
+def test_attention_matches_fp64(impl, Hq, Hkv, Dh, L, cache_seq, nbs):
     B = len(nbs)
     rows = sum(nbs)
     row_off = np.concatenate([[0], np.cumsum(nbs)]).astype(np.int32)
     ldq = (Hq + 2 * Hkv) * Dh                                          # Q sits inside a wider QKV row, as in the step
     q = _bf16((rows + 3, ldq), 5)
     kc = _bf16((B, cache_seq, Hkv, Dh), 6); vc = _bf16((B, cache_seq, Hkv, Dh), 7)
-    o, lse, abar = binding.d2c_op_attention(q.cuda(), kc.cuda(), vc.cuda(), torch.from_numpy(row_off).cuda(), L, Hq, Hkv, Dh)
+    o, lse, abar = binding.d2c_op_attention(q.cuda(), kc.cuda(), vc.cuda(), torch.from_numpy(row_off).cuda(), L, Hq, Hkv, Dh,
+                                            impl=impl)
     torch.cuda.synchronize()
     wo, wl, wa = _attention_ref(q.double().numpy()[:rows], kc.double().numpy(), vc.double().numpy(), row_off, L, Hq, Hkv, Dh)
     assert row_rel_err(o.float().cpu().numpy()[:rows], wo) <= ROW_TOL
