@@ -179,7 +179,7 @@ int d2c_sync_status(d2c_ctx* ctx);
  * milliseconds spent in each phase (phase_ms[D2C_N_PHASES]) and the number of kernels the library
  * launched in it (phase_launches[D2C_N_PHASES]); either may be NULL.  d2c_phase_name(i) names
  * phase i ("select", "gemm_qkv", ...). */
-#define D2C_N_PHASES 12
+#define D2C_N_PHASES 13
 int d2c_profile(d2c_ctx* ctx, int32_t enable);
 int d2c_profile_read(d2c_ctx* ctx, float* phase_ms, int64_t* phase_launches, int32_t reset);
 const char* d2c_phase_name(int32_t i);

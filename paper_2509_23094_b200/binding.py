@@ -14,7 +14,7 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libd2c.so")
 
-N_PHASES = 12
+N_PHASES = 13
 D2C_OK, D2C_EINVAL, D2C_ESHAPE, D2C_ECAPACITY, D2C_ECUDA, D2C_ETIMEOUT = 0, -1, -2, -3, -4, -5
 
 # every symbol include/d2c.h declares

@@ -255,9 +255,11 @@ int launch_dh(const AttnArgs& a, cudaStream_t st) {
     attr_set = true;
   }
   const int qtiles = ceil_div(a.max_rows_per_seq, QT);
-  attn_fwd_kernel<DH><<<dim3(qtiles, a.hq, a.batch), ATHREADS, smem_fwd, st>>>(a);
-  D2C_LAUNCHED();
-  if (a.abar) {
+  if (a.which != 2) {
+    attn_fwd_kernel<DH><<<dim3(qtiles, a.hq, a.batch), ATHREADS, smem_fwd, st>>>(a);
+    D2C_LAUNCHED();
+  }
+  if (a.abar && a.which != 1) {
     attn_abar_kernel<DH><<<dim3(ceil_div(a.seq_len, KT), qtiles, a.batch), ATHREADS, smem_ab, st>>>(a);
     D2C_LAUNCHED();
   }

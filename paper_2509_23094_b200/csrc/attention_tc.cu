@@ -1,17 +1,16 @@
 // Selected-query bidirectional attention on the 5th-generation tensor cores (head_dim 128).
 //
 //   attn_fwd_tc    O = softmax(Q K^T / sqrt(Dh)) V and the log-sum-exp per (row, head).  One CTA per
-//                  (128 selected rows, head, sequence); keys stream in tiles of 128 through TMA.
-//                  S = Q K^T is a tcgen05.mma into TMEM; four softmax warps (one row per thread) read it
+//                  (256 selected rows, head, sequence); keys stream in tiles of 128 through TMA.
+//                  S = Q K^T is a tcgen05.mma into TMEM; softmax warps (one row per thread) read it
 //                  with tcgen05.ld, write the bf16 probabilities back over the same TMEM columns and the
 //                  PV product takes them from there as its A operand (V is the MN-major B operand straight
-//                  from the TMA tile).  Each tile's PV lands in its own TMEM buffer and is folded into
-//                  fp32 registers with the usual running-max rescale, so no TMEM read-modify-write exists.
+//                  from the TMA tile) and accumulates O in TMEM.
 //   attn_abar_tc   Abar[r][j] = 1/Hq sum_h exp(s_h[r][j] - lse_h[r]) (Section 4.2): one CTA per
 //                  (128 rows x 128 keys) loops over the heads, S by tcgen05.mma, the sum over heads in
 //                  registers in a fixed order (deterministic).
 //
-// Warp roles in both: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-5 softmax/epilogue.
+// Warp roles in both: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2.. softmax/epilogue.
 // No cluster, no multicast.  Every mbarrier wait is bounded (see gemm_tc.cu for the protocol).
 #include <cuda.h>
 
@@ -127,24 +126,44 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 struct AttnTcParams { AttnArgs a; int* status; };
 
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(ATC_THREADS, 1)
+// Forward kernel.  One CTA owns up to 256 selected rows of one (sequence, head): two query tiles of
+// 128 rows that share every K/V tile brought in by TMA.  Each query tile has its own softmax warp
+// group (4 warps, one row per thread) and its own TMEM columns: 128 for the scores S (overwritten in
+// place by the bf16 probabilities P) and 128 for the output accumulator O, which stays in TMEM across
+// the key tiles.  The running maximum is only raised when it grows by more than 2^8 (P stays exactly
+// representable in bf16's exponent range); the rare raise rescales O in TMEM between two PV products.
+constexpr int FWD_THREADS = 320;
+constexpr float kRescaleStep = 8.f;
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+               "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+               ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                 "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+                 "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+                 "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+}
+
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
   const AttnArgs& a = p.a;
   const int b = blockIdx.z, h = blockIdx.y, g = h / (a.hq / a.hkv);
-  const int r0 = a.row_off[b] + blockIdx.x * AQ;
-  const int nrows = min(AQ, a.row_off[b + 1] - r0);
+  const int r0 = a.row_off[b] + blockIdx.x * 2 * AQ;
+  const int nrows = min(2 * AQ, a.row_off[b + 1] - r0);
   if (nrows <= 0) return;                                          // uniform: nothing allocated yet
+  const int nq = nrows > AQ ? 2 : 1;                                // live query tiles
   const int L = a.seq_len, T = (L + AKEYS - 1) / AKEYS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int* status = p.status ? p.status : g_attn_status;
 
   extern __shared__ unsigned char smem_raw[];
-  const uint32_t sQ = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
-  auto sK = [&](int s) { return sQ + TILE_BYTES + s * 2 * TILE_BYTES; };
-  auto sV = [&](int s) { return sK(s) + TILE_BYTES; };
-  // barriers: 0 q_full | 1,2 k_full | 3,4 v_full | 5,6 kv_empty | 7,8 s_full | 9,10 p_full | 11,12 o_full | 13,14 o_empty
-  __shared__ __align__(8) uint64_t bars[15];
+  const uint32_t sbase = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
+  auto sQ = [&](int q) { return sbase + q * TILE_BYTES; };
+  auto sK = [&](int s) { return sbase + (2 + 2 * s) * TILE_BYTES; };
+  auto sV = [&](int s) { return sbase + (3 + 2 * s) * TILE_BYTES; };
+  // barriers: 0 q_full | 1,2 k_full | 3,4 v_full | 5,6 kv_empty | 7,8 s_full[q] | 9,10 p_full[q] | 11,12 o_full[q]
+  __shared__ __align__(8) uint64_t bars[13];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
@@ -153,7 +172,6 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     for (int i = 0; i < 9; ++i) mbar_init(B(i), 1);
     mbar_init(B(9), 4); mbar_init(B(10), 4);
     mbar_init(B(11), 1); mbar_init(B(12), 1);
-    mbar_init(B(13), 4); mbar_init(B(14), 4);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -162,15 +180,17 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tm = tmem_slot;                                    // S/P buffers at +0, +128; PV buffers at +256, +384
+  const uint32_t tm = tmem_slot;                                    // tile q: S/P at q*256, O at q*256 + 128
   volatile int* abortp = &abort_flag;
   const int kv_row0 = b * a.cache_seq;
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(B(0), TILE_BYTES);
-      tma_load_2d(sQ, &tmQ, h * ADH, r0, B(0));
-      tma_load_2d(sQ + HALF_BYTES, &tmQ, h * ADH + 64, r0, B(0));
+      mbar_expect_tx(B(0), nq * TILE_BYTES);
+      for (int q = 0; q < nq; ++q) {
+        tma_load_2d(sQ(q), &tmQ, h * ADH, r0 + q * AQ, B(0));
+        tma_load_2d(sQ(q) + HALF_BYTES, &tmQ, h * ADH + 64, r0 + q * AQ, B(0));
+      }
       int issued = 0;
       for (int j = 0; j < T; ++j) {
         const int s = j & 1, u = j >> 1;
@@ -196,114 +216,138 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
-      bool ok = mbar_wait(B(0), 0, abortp, status, 12);
-      auto issue_s = [&](int j) {                                   // S_j = Q K_j^T into buffer j & 1
+      auto issue_s = [&](int q, int j) {                            // S_{q,j} = Q_q K_j^T
         const int s = j & 1;
-        if (!mbar_wait(B(1 + s), (j >> 1) & 1, abortp, status, 13)) return false;
-        tc_fence_after();
 #pragma unroll
         for (int i = 0; i < ADH / 16; ++i) {
           const uint32_t off = (i >> 2) * HALF_BYTES;
-          umma_ss(tm + s * 128, desc_kmajor(sQ + off) + 2 * (i & 3), desc_kmajor(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
+          umma_ss(tm + q * 256, desc_kmajor(sQ(q) + off) + 2 * (i & 3), desc_kmajor(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
         }
-        umma_commit(B(7 + s));
-        return true;
+        umma_commit(B(7 + q));
       };
-      if (ok) ok = issue_s(0);
+      bool ok = mbar_wait(B(0), 0, abortp, status, 12) && mbar_wait(B(1), 0, abortp, status, 13);
+      if (ok) {
+        tc_fence_after();
+        for (int q = 0; q < nq; ++q) issue_s(q, 0);
+      }
       for (int j = 0; j < T && ok; ++j) {
         const int s = j & 1, u = j >> 1;
-        if (j + 1 < T) { ok = issue_s(j + 1); if (!ok) break; }
-        if (!mbar_wait(B(9 + s), u & 1, abortp, status, 14) || !mbar_wait(B(3 + s), u & 1, abortp, status, 15) ||
-            !mbar_wait(B(13 + s), (u & 1) ^ 1, abortp, status, 16)) { ok = false; break; }
-        tc_fence_after();
+        for (int q = 0; q < nq && ok; ++q) {
+          if (!mbar_wait(B(9 + q), j & 1, abortp, status, 14)) { ok = false; break; }
+          if (q == 0 && !mbar_wait(B(3 + s), u & 1, abortp, status, 15)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int i = 0; i < AKEYS / 16; ++i)                       // P_j (TMEM, 8 columns per 16 keys) x V_j
-          umma_ts(tm + 256 + s * 128, tm + s * 128 + 8 * i, desc_mnmajor(sV(s) + i * 2048), kIdescKMn, i != 0);
-        umma_commit(B(5 + s));                                      // K/V stage free
-        umma_commit(B(11 + s));                                     // PV_j ready
+          for (int i = 0; i < AKEYS / 16; ++i)                     // O_q += P_{q,j} (TMEM, 8 columns per 16 keys) x V_j
+            umma_ts(tm + q * 256 + 128, tm + q * 256 + 8 * i, desc_mnmajor(sV(s) + i * 2048), kIdescKMn, (j | i) != 0);
+          umma_commit(B(11 + q));
+          if (q == nq - 1) umma_commit(B(5 + s));                   // both products of tile j issued: K/V stage free when done
+          if (j + 1 < T) {
+            if (q == 0 && !mbar_wait(B(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abortp, status, 16)) { ok = false; break; }
+            tc_fence_after();
+            issue_s(q, j + 1);                                      // after PV_{q,j} in program order: P_{q,j} is consumed first
+          }
+        }
       }
     }
     __syncwarp();
   } else {
-    const int quarter = warp & 3, lrow = quarter * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const float sc = kLog2e * rsqrtf((float)ADH);
-    float o[ADH];
+    const int q = (warp - 2) >> 2;                                  // softmax warp group = query tile
+    if (q < nq) {
+      const int quarter = warp & 3, lrow = q * AQ + quarter * 32 + lane;
+      const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+      const uint32_t ts = tm + q * 256 + lane_base, to = ts + 128;
+      const float sc = kLog2e * rsqrtf((float)ADH);
+      float m_used = -INFINITY, l = 0.f;
+      bool ok = true;
+      for (int j = 0; j < T && ok; ++j) {
+        if (!mbar_wait(B(7 + q), j & 1, abortp, status, 18)) { ok = false; break; }
+        tc_fence_after();
+        const int key0 = j * AKEYS;
+        const bool full = key0 + AKEYS <= L;
+        uint32_t sv[4][32];                                         // the whole score row of this thread
 #pragma unroll
-    for (int i = 0; i < ADH; ++i) o[i] = 0.f;
-    float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
-    bool ok = true;
-    auto fold_pv = [&](int j, float alpha) {                        // o = o * alpha + PV_j
-      const int s = j & 1;
-      if (!mbar_wait(B(11 + s), (j >> 1) & 1, abortp, status, 17)) return false;
-      tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tm + 256 + s * 128 + lane_base + c * 32, v);
+        for (int c = 0; c < 4; ++c) tmem_ld32(ts + c * 32, sv[c]);
         tmem_ld_wait();
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(v[i]));
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(B(13 + s));
-      return true;
-    };
-    for (int j = 0; j < T && ok; ++j) {
-      const int s = j & 1;
-      if (!mbar_wait(B(7 + s), (j >> 1) & 1, abortp, status, 18)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t ts = tm + s * 128 + lane_base;
-      const int key0 = j * AKEYS;
-      float mx = m;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {                                 // pass 1: running maximum
-        uint32_t v[32];
-        tmem_ld32(ts + c * 32, v);
-        tmem_ld_wait();
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (key0 + c * 32 + i < L) mx = fmaxf(mx, __uint_as_float(v[i]) * sc);
-      }
-      const float alpha = exp2f(m - mx);                            // first tile: exp2(-inf) = 0
-      m = mx;
-      float rs = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {                                 // pass 2: probabilities, written back as bf16
-        uint32_t v[32], pk[16];
-        tmem_ld32(ts + c * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int k = key0 + c * 32 + 2 * i;
-          const float p0 = k < L ? exp2f(__uint_as_float(v[2 * i]) * sc - m) : 0.f;
-          const float p1 = k + 1 < L ? exp2f(__uint_as_float(v[2 * i + 1]) * sc - m) : 0.f;
-          rs += p0 + p1;
-          pk[i] = pack_bf16(p0, p1);
+          for (int i = 0; i < 32; ++i) {
+            const float f = __uint_as_float(sv[c][i]);
+            if (full || key0 + c * 32 + i < L) mx4[i & 3] = fmaxf(mx4[i & 3], f);
+          }
         }
-        tmem_st16(ts + c * 16, pk);                                 // lands on columns whose scores are already consumed
-      }
-      l = l * alpha + rs;
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(B(9 + s));
-      if (j >= 1) ok = fold_pv(j - 1, alpha_prev);
-      alpha_prev = alpha;
-    }
-    if (ok) ok = fold_pv(T - 1, alpha_prev);
-    if (ok && lrow < nrows) {
-      const float inv = 1.f / l;
-      bf16* dst = a.o + (size_t)(r0 + lrow) * ((size_t)a.hq * ADH) + (size_t)h * ADH;
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+        const bool raise = mx > m_used + kRescaleStep;              // always true on the first tile
+        if (__any_sync(0xffffffffu, raise)) {
+          const float alpha = raise ? exp2f(m_used - mx) : 1.f;     // first tile: exp2(-inf) = 0
+          if (raise) m_used = mx;
+          l *= alpha;
+          if (j > 0) {                                              // O holds the sum of tiles 0..j-1: rescale it in place
+            if (!mbar_wait(B(11 + q), (j - 1) & 1, abortp, status, 17)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t v[32];
+              tmem_ld32(to + c * 32, v);
+              tmem_ld_wait();
 #pragma unroll
-      for (int q = 0; q < ADH / 8; ++q) {
-        uint4 w;
-        w.x = pack_bf16(o[q * 8 + 0] * inv, o[q * 8 + 1] * inv); w.y = pack_bf16(o[q * 8 + 2] * inv, o[q * 8 + 3] * inv);
-        w.z = pack_bf16(o[q * 8 + 4] * inv, o[q * 8 + 5] * inv); w.w = pack_bf16(o[q * 8 + 6] * inv, o[q * 8 + 7] * inv);
-        reinterpret_cast<uint4*>(dst)[q] = w;
+              for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+              tmem_st32(to + c * 32, v);
+            }
+            tmem_st_wait();
+          }
+        }
+        float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {                               // probabilities, written back as bf16 over the scores
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = exp2f(fmaf(__uint_as_float(sv[c][2 * i]), sc, -m_used));
+            float p1 = exp2f(fmaf(__uint_as_float(sv[c][2 * i + 1]), sc, -m_used));
+            if (!full) {
+              const int k = key0 + c * 32 + 2 * i;
+              if (k >= L) p0 = 0.f;
+              if (k + 1 >= L) p1 = 0.f;
+            }
+            rs4[i & 3] += p0 + p1;
+            pk[i] = pack_bf16(p0, p1);
+          }
+          tmem_st16(ts + c * 16, pk);
+        }
+        const float rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+        l += rs;
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(B(9 + q));
       }
-      a.lse[(size_t)(r0 + lrow) * a.hq + h] = (m + log2f(l)) * kLn2;
+      if (ok) ok = mbar_wait(B(11 + q), (T - 1) & 1, abortp, status, 19);
+      tc_fence_after();
+      if (ok) {
+        const bool row_ok = lrow < nrows;
+        const float inv = 1.f / l;
+        bf16* dst = a.o + (size_t)(r0 + lrow) * ((size_t)a.hq * ADH) + (size_t)h * ADH;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t v[32];
+          tmem_ld32(to + c * 32, v);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(v[8 * t + 0]) * inv, __uint_as_float(v[8 * t + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(v[8 * t + 2]) * inv, __uint_as_float(v[8 * t + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(v[8 * t + 4]) * inv, __uint_as_float(v[8 * t + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(v[8 * t + 6]) * inv, __uint_as_float(v[8 * t + 7]) * inv);
+              reinterpret_cast<uint4*>(dst)[c * 4 + t] = w;
+            }
+          }
+        }
+        if (row_ok) a.lse[(size_t)(r0 + lrow) * a.hq + h] = (m_used + log2f(l)) * kLn2;
+      }
     }
   }
   tc_fence_before();
@@ -312,7 +356,9 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 }
 
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(ATC_THREADS, 1)
+constexpr int ABS = 3;                             // stages of the Q ring and of the K ring in attn_abar_tc
+
+__global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const AttnTcParams p) {
   const AttnArgs& a = p.a;
   const int b = blockIdx.z;
@@ -326,17 +372,22 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
-  auto sQ = [&](int s) { return base + s * TILE_BYTES; };           // two Q stages, then two K stages
-  auto sK = [&](int s) { return base + (2 + s) * TILE_BYTES; };
-  // barriers: 0,1 q_full | 2,3 k_full | 4,5 q_empty | 6,7 k_empty | 8,9 s_full | 10,11 s_empty
-  __shared__ __align__(8) uint64_t bars[12];
+  auto sQ = [&](int s) { return base + s * TILE_BYTES; };           // ABS query stages, then ABS key stages
+  auto sK = [&](int s) { return base + (ABS + s) * TILE_BYTES; };
+  // barriers: q_full[ABS] | k_full[ABS] | q_empty[ABS] | k_empty[ABS] | s_full[2] | s_empty[2]
+  __shared__ __align__(8) uint64_t bars[4 * ABS + 4];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
-  auto B = [&](int i) { return bar0 + 8u * i; };
+  auto QF = [&](int i) { return bar0 + 8u * i; };
+  auto KF = [&](int i) { return bar0 + 8u * (ABS + i); };
+  auto QE = [&](int i) { return bar0 + 8u * (2 * ABS + i); };
+  auto KE = [&](int i) { return bar0 + 8u * (3 * ABS + i); };
+  auto SF = [&](int i) { return bar0 + 8u * (4 * ABS + i); };
+  auto SE = [&](int i) { return bar0 + 8u * (4 * ABS + 2 + i); };
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 10; ++i) mbar_init(B(i), 1);
-    mbar_init(B(10), 4); mbar_init(B(11), 4);
+    for (int i = 0; i < 4 * ABS + 2; ++i) mbar_init(bar0 + 8u * i, 1);
+    mbar_init(SE(0), 8); mbar_init(SE(1), 8);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -353,24 +404,24 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (lane == 0) {
       int issued = 0;
       for (int h = 0; h < a.hq; ++h) {
-        const int s = h & 1, u = h >> 1;
-        if (!mbar_wait(B(4 + s), (u & 1) ^ 1, abortp, status, 21)) break;
-        mbar_expect_tx(B(s), TILE_BYTES);
-        tma_load_2d(sQ(s), &tmQ, h * ADH, r0, B(s));
-        tma_load_2d(sQ(s) + HALF_BYTES, &tmQ, h * ADH + 64, r0, B(s));
+        const int s = h % ABS, u = h / ABS;
+        if (!mbar_wait(QE(s), (u & 1) ^ 1, abortp, status, 21)) break;
+        mbar_expect_tx(QF(s), TILE_BYTES);
+        tma_load_2d(sQ(s), &tmQ, h * ADH, r0, QF(s));
+        tma_load_2d(sQ(s) + HALF_BYTES, &tmQ, h * ADH + 64, r0, QF(s));
         if (h % group == 0) {
-          const int gi = h / group, ks = gi & 1, ku = gi >> 1;
-          if (!mbar_wait(B(6 + ks), (ku & 1) ^ 1, abortp, status, 22)) break;
-          mbar_expect_tx(B(2 + ks), TILE_BYTES);
-          tma_load_2d(sK(ks), &tmK, gi * ADH, kv_row, B(2 + ks));
-          tma_load_2d(sK(ks) + HALF_BYTES, &tmK, gi * ADH + 64, kv_row, B(2 + ks));
+          const int gi = h / group, ks = gi % ABS, ku = gi / ABS;
+          if (!mbar_wait(KE(ks), (ku & 1) ^ 1, abortp, status, 22)) break;
+          mbar_expect_tx(KF(ks), TILE_BYTES);
+          tma_load_2d(sK(ks), &tmK, gi * ADH, kv_row, KF(ks));
+          tma_load_2d(sK(ks) + HALF_BYTES, &tmK, gi * ADH + 64, kv_row, KF(ks));
         }
         issued = h + 1;
       }
       if (*abortp) {
-        for (int h = max(0, issued - 2); h < issued; ++h) {
+        for (int h = max(0, issued - ABS); h < issued; ++h) {
           const long long t1 = clock64();
-          while (!mbar_try_wait(B(h & 1), (h >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
+          while (!mbar_try_wait(QF(h % ABS), (h / ABS) & 1) && clock64() - t1 < kWaitCycles) {}
         }
       }
     }
@@ -378,59 +429,62 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   } else if (warp == 1) {
     if (lane == 0) {
       for (int h = 0; h < a.hq; ++h) {
-        const int s = h & 1, u = h >> 1, gi = h / group, ks = gi & 1, ku = gi >> 1;
-        if (!mbar_wait(B(s), u & 1, abortp, status, 23)) break;
-        if (h % group == 0 && !mbar_wait(B(2 + ks), ku & 1, abortp, status, 24)) break;
-        if (!mbar_wait(B(10 + s), (u & 1) ^ 1, abortp, status, 25)) break;
+        const int s = h % ABS, u = h / ABS, gi = h / group, ks = gi % ABS, ku = gi / ABS, sb = h & 1;
+        if (!mbar_wait(QF(s), u & 1, abortp, status, 23)) break;
+        if (h % group == 0 && !mbar_wait(KF(ks), ku & 1, abortp, status, 24)) break;
+        if (!mbar_wait(SE(sb), ((h >> 1) & 1) ^ 1, abortp, status, 25)) break;
         tc_fence_after();
 #pragma unroll
         for (int i = 0; i < ADH / 16; ++i) {
           const uint32_t off = (i >> 2) * HALF_BYTES;
-          umma_ss(tm + s * 128, desc_kmajor(sQ(s) + off) + 2 * (i & 3), desc_kmajor(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
+          umma_ss(tm + sb * 128, desc_kmajor(sQ(s) + off) + 2 * (i & 3), desc_kmajor(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
         }
-        umma_commit(B(4 + s));                                      // Q stage free
-        if ((h + 1) % group == 0 || h + 1 == a.hq) umma_commit(B(6 + ks));   // last head of the group: K stage free
-        umma_commit(B(8 + s));
+        umma_commit(QE(s));                                         // Q stage free
+        if ((h + 1) % group == 0 || h + 1 == a.hq) umma_commit(KE(ks));      // last head of the group: K stage free
+        umma_commit(SF(sb));
       }
     }
     __syncwarp();
   } else {
-    const int quarter = warp & 3, lrow = quarter * 32 + lane;
+    // eight warps: two per TMEM lane quarter, each owning 64 of the tile's 128 key columns, so that the
+    // two warps of a scheduler hide each other's TMEM-load latency
+    const int quarter = warp & 3, half = (warp - 2) >> 2, lrow = quarter * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const float sc = kLog2e * rsqrtf((float)ADH);
     const bool row_ok = lrow < nrows;
-    float acc[AKEYS];
+    float acc[64];
 #pragma unroll
-    for (int i = 0; i < AKEYS; ++i) acc[i] = 0.f;
+    for (int i = 0; i < 64; ++i) acc[i] = 0.f;
     bool ok = true;
     for (int h = 0; h < a.hq && ok; ++h) {
-      const int s = h & 1;
+      const int sb = h & 1;
       const float e = row_ok ? a.lse[(size_t)(r0 + lrow) * a.hq + h] * kLog2e : 0.f;
-      if (!mbar_wait(B(8 + s), (h >> 1) & 1, abortp, status, 26)) { ok = false; break; }
+      if (!mbar_wait(SF(sb), (h >> 1) & 1, abortp, status, 26)) { ok = false; break; }
       tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tm + s * 128 + lane_base + c * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) acc[c * 32 + i] += exp2f(__uint_as_float(v[i]) * sc - e);
-      }
+      uint32_t v[2][32];
+      tmem_ld32(tm + sb * 128 + lane_base + half * 64, v[0]);
+      tmem_ld32(tm + sb * 128 + lane_base + half * 64 + 32, v[1]);
+      tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(B(10 + s));
+      if (lane == 0) mbar_arrive(SE(sb));                           // scores are in registers: the buffer may be refilled
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[c * 32 + i] += exp2f(fmaf(__uint_as_float(v[c][i]), sc, -e));
     }
     if (ok && row_ok) {
       const float inv = 1.f / (float)a.hq;
-      float* dst = a.abar + (size_t)(r0 + lrow) * L + key0;
-      if (key0 + AKEYS <= L && (L & 3) == 0) {
+      const int k0 = key0 + half * 64;
+      float* dst = a.abar + (size_t)(r0 + lrow) * L + k0;
+      if (k0 + 64 <= L && (L & 3) == 0) {
 #pragma unroll
-        for (int q = 0; q < AKEYS / 4; ++q)
+        for (int q = 0; q < 16; ++q)
           reinterpret_cast<float4*>(dst)[q] = make_float4(acc[4 * q] * inv, acc[4 * q + 1] * inv, acc[4 * q + 2] * inv, acc[4 * q + 3] * inv);
       } else {
 #pragma unroll
-        for (int i = 0; i < AKEYS; ++i)
-          if (key0 + i < L) dst[i] = acc[i] * inv;
+        for (int i = 0; i < 64; ++i)
+          if (k0 + i < L) dst[i] = acc[i] * inv;
       }
     }
   }
@@ -477,7 +531,7 @@ bool attention_tc_supported(const AttnArgs& a) {
 }
 
 int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
-  const int smem_fwd = 5 * TILE_BYTES + 1024, smem_ab = 4 * TILE_BYTES + 1024;
+  const int smem_fwd = 6 * TILE_BYTES + 1024, smem_ab = 2 * ABS * TILE_BYTES + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     D2C_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_fwd));
@@ -492,10 +546,12 @@ int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   if (rc != D2C_OK) return rc;
   AttnTcParams p{a, status};
   const int qtiles = ceil_div(a.max_rows_per_seq, AQ);
-  attn_fwd_tc<<<dim3(qtiles, a.hq, a.batch), ATC_THREADS, smem_fwd, st>>>(tmQ, tmK, tmV, p);
-  D2C_LAUNCHED();
-  if (a.abar) {
-    attn_abar_tc<<<dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), ATC_THREADS, smem_ab, st>>>(tmQ, tmK, p);
+  if (a.which != 2) {
+    attn_fwd_tc<<<dim3(ceil_div(a.max_rows_per_seq, 2 * AQ), a.hq, a.batch), FWD_THREADS, smem_fwd, st>>>(tmQ, tmK, tmV, p);
+    D2C_LAUNCHED();
+  }
+  if (a.abar && a.which != 1) {
+    attn_abar_tc<<<dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), FWD_THREADS, smem_ab, st>>>(tmQ, tmK, p);
     D2C_LAUNCHED();
   }
   return D2C_OK;

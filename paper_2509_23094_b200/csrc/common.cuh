@@ -80,6 +80,7 @@ struct AttnArgs {
   int q_rows;                            // rows the q buffer holds (bounds the TMA map)
   int portable;                          // 1: force the mma.sync kernels
   int* status;                           // device status word for bounded waits (may be null)
+  int which;                             // 0: both kernels, 1: O/LSE only, 2: head-averaged probabilities only
 };
 int launch_attention(const AttnArgs& a, cudaStream_t st);
 bool attention_tc_supported(const AttnArgs& a);               // attention_tc.cu

@@ -22,8 +22,8 @@ void count_launch(int n) { g_launches += n; }
 
 static const char* const kPhaseNames[D2C_N_PHASES] = {
     "select", "gather_norm", "rmsnorm", "gemm_qkv", "rope_scatter", "attention", "gemm_o",
-    "gemm_gate_up", "gemm_down", "lm_head", "rollout", "copy_out"};
-enum Phase { PH_SELECT = 0, PH_GATHER, PH_NORM, PH_QKV, PH_ROPE, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM, PH_ROLLOUT, PH_OUT };
+    "gemm_gate_up", "gemm_down", "lm_head", "rollout", "copy_out", "attn_abar"};
+enum Phase { PH_SELECT = 0, PH_GATHER, PH_NORM, PH_QKV, PH_ROPE, PH_ATTN, PH_O, PH_GATEUP, PH_DOWN, PH_LM, PH_ROLLOUT, PH_OUT, PH_ABAR };
 
 // Hands out 256-byte aligned pieces of a buffer; with base == null it only measures.
 struct Carver {
@@ -299,7 +299,13 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     at.q_rows = R; at.portable = (c.flags & D2C_FLAG_PORTABLE_ATTENTION) ? 1 : 0; at.status = b.status;
     at.o = b.o; at.lse = b.lse; at.abar = l < depth ? b.abar + (size_t)l * c.max_batch * c.max_seq * c.max_seq : nullptr;
     D2C_TRY(ctx, mark(ctx, PH_ATTN));
+    at.which = 1;
     D2C_TRY(ctx, launch_attention(at, st));
+    if (at.abar) {
+      D2C_TRY(ctx, mark(ctx, PH_ABAR));
+      at.which = 2;
+      D2C_TRY(ctx, launch_attention(at, st));
+    }
     D2C_TRY(ctx, mark(ctx, PH_O));
     GemmArgs go{};
     go.A = b.o; go.lda = hq * dh; go.W = ctx->wo[l]; go.C = x; go.ldc = d; go.n_rows = n_rows; go.max_rows = R; go.N = d; go.K = hq * dh;
