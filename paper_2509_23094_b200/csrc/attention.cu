@@ -59,6 +59,7 @@ __device__ __forceinline__ void load_tile(uint32_t sdst, const bf16* src, size_t
 
 template <int DH>
 __global__ void __launch_bounds__(ATHREADS) attn_fwd_kernel(AttnArgs a) {
+  pdl_prologue();
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int TILE = KT * DH * 2;
   const int b = blockIdx.z, h = blockIdx.y, g = h / (a.hq / a.hkv);
@@ -174,6 +175,7 @@ __global__ void __launch_bounds__(ATHREADS) attn_fwd_kernel(AttnArgs a) {
 
 template <int DH>
 __global__ void __launch_bounds__(ATHREADS) attn_abar_kernel(AttnArgs a) {
+  pdl_prologue();
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int TILE = KT * DH * 2;
   const int b = blockIdx.z;
@@ -256,12 +258,10 @@ int launch_dh(const AttnArgs& a, cudaStream_t st) {
   }
   const int qtiles = ceil_div(a.max_rows_per_seq, QT);
   if (a.which != 2) {
-    attn_fwd_kernel<DH><<<dim3(qtiles, a.hq, a.batch), ATHREADS, smem_fwd, st>>>(a);
-    D2C_LAUNCHED();
+    D2C_LAUNCH((attn_fwd_kernel<DH>), dim3(qtiles, a.hq, a.batch), ATHREADS, smem_fwd, st, a);
   }
   if (a.abar && a.which != 1) {
-    attn_abar_kernel<DH><<<dim3(ceil_div(a.seq_len, KT), qtiles, a.batch), ATHREADS, smem_ab, st>>>(a);
-    D2C_LAUNCHED();
+    D2C_LAUNCH((attn_abar_kernel<DH>), dim3(ceil_div(a.seq_len, KT), qtiles, a.batch), ATHREADS, smem_ab, st, a);
   }
   return D2C_OK;
 }

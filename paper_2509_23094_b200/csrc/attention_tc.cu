@@ -147,6 +147,7 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const AttnTcParams p) {
+  pdl_prologue();
   const AttnArgs& a = p.a;
   const int b = blockIdx.z, h = blockIdx.y, g = h / (a.hq / a.hkv);
   const int r0 = a.row_off[b] + blockIdx.x * 2 * AQ;
@@ -360,6 +361,7 @@ constexpr int ABS = 3;                             // stages of the Q ring and o
 
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const AttnTcParams p) {
+  pdl_prologue();
   const AttnArgs& a = p.a;
   const int b = blockIdx.z;
   const int r0 = a.row_off[b] + blockIdx.y * AQ;
@@ -547,12 +549,10 @@ int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   AttnTcParams p{a, status};
   const int qtiles = ceil_div(a.max_rows_per_seq, AQ);
   if (a.which != 2) {
-    attn_fwd_tc<<<dim3(ceil_div(a.max_rows_per_seq, 2 * AQ), a.hq, a.batch), FWD_THREADS, smem_fwd, st>>>(tmQ, tmK, tmV, p);
-    D2C_LAUNCHED();
+    D2C_LAUNCH((attn_fwd_tc), dim3(ceil_div(a.max_rows_per_seq, 2 * AQ), a.hq, a.batch), FWD_THREADS, smem_fwd, st, tmQ, tmK, tmV, p);
   }
   if (a.abar && a.which != 1) {
-    attn_abar_tc<<<dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), FWD_THREADS, smem_ab, st>>>(tmQ, tmK, p);
-    D2C_LAUNCHED();
+    D2C_LAUNCH((attn_abar_tc), dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), FWD_THREADS, smem_ab, st, tmQ, tmK, p);
   }
   return D2C_OK;
 }

@@ -12,6 +12,7 @@ struct CommitArgs {
 };
 
 __global__ void __launch_bounds__(256) commit_kernel(CommitArgs a) {
+  pdl_prologue();
   extern __shared__ unsigned char take[];                       // [seq_len] 1 = commit this position
   __shared__ unsigned long long s_best[8];
   const int b = blockIdx.x, L = a.seq_len, tid = threadIdx.x;
@@ -64,8 +65,7 @@ int launch_commit(int batch, int seq_len, int d, int rule, float threshold, cons
                   const float* conf, const int32_t* pred, const uint32_t* phi, int phi_len, const bf16* embed,
                   bf16* h0, uint8_t* mask, int32_t* tokens, int32_t* committed, cudaStream_t st) {
   CommitArgs a{seq_len, d, rule, threshold, slot_of_pos, conf, pred, phi, phi_len, embed, h0, mask, tokens, committed};
-  commit_kernel<<<batch, 256, seq_len, st>>>(a);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((commit_kernel), batch, 256, seq_len, st, a);
   return D2C_OK;
 }
 

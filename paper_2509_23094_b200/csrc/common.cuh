@@ -28,6 +28,30 @@ void count_launch(int n);
       return D2C_ECUDA;                                                                \
     }                                                                                  \
   } while (0)
+// Programmatic dependent launch: every kernel of the step is launched with the stream-serialisation
+// attribute and starts with pdl_prologue(), which waits for the preceding kernel's results and then
+// lets the following kernel begin its own launch, so launch latency overlaps the predecessor's tail.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+#define D2C_LAUNCH(kernel, grid, block, smem, st, ...)                                      \
+  do {                                                                                      \
+    D2C_CUDA_OK(d2c::launch_pdl(kernel, grid, block, smem, st, __VA_ARGS__));               \
+    d2c::count_launch(1);                                                                   \
+  } while (0)
 // After a kernel launch: checks the launch and counts it.
 #define D2C_LAUNCHED() do { D2C_CUDA_OK(cudaGetLastError()); d2c::count_launch(1); } while (0)
 

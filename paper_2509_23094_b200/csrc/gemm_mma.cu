@@ -49,6 +49,7 @@ __device__ __forceinline__ void b_row_source(int r, int tile_n, int& col, bool& 
 
 template <int EPI>
 __global__ void __launch_bounds__(THREADS, 2) gemm_mma_kernel(GemmArgs g) {
+  pdl_prologue();
   extern __shared__ __align__(128) unsigned char smem[];
   const int n = *g.n_rows;
   const int m0 = blockIdx.y * BM;
@@ -230,8 +231,7 @@ int launch_one(const GemmArgs& g, cudaStream_t st) {
   }
   const int n_tiles = EPI == EPI_SWIGLU ? ceil_div(g.N, 64) : ceil_div(g.N, BN);
   dim3 grid(n_tiles, ceil_div(g.max_rows, BM));
-  gemm_mma_kernel<EPI><<<grid, THREADS, smem, st>>>(g);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((gemm_mma_kernel<EPI>), grid, THREADS, smem, st, g);
   return D2C_OK;
 }
 }  // namespace

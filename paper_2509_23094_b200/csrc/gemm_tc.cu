@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant__ CUtensorMap tmA64,
                const __grid_constant__ CUtensorMap tmA32, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  pdl_prologue();
   constexpr int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : 256;  // output columns per tile
   const GemmArgs& g = p.g;
   const int n = *g.n_rows;
@@ -427,8 +428,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   const int out_cols = EPI == EPI_SWIGLU ? 128 : 256;
   const long long tiles = (long long)ceil_div(g.max_rows, TM) * ceil_div(g.N, out_cols);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  gemm_tc_kernel<EPI><<<grid, TC_THREADS, smem, st>>>(tmA128, tmA64, tmA32, tmB, tmB2, p);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((gemm_tc_kernel<EPI>), grid, TC_THREADS, smem, st, tmA128, tmA64, tmA32, tmB, tmB2, p);
   return D2C_OK;
 }
 }  // namespace

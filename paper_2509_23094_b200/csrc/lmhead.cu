@@ -13,6 +13,7 @@ lm_reduce_kernel(const float* __restrict__ st_max, const float* __restrict__ st_
                  const int32_t* __restrict__ lm_rows, const int32_t* __restrict__ sel_idx,
                  const int32_t* __restrict__ row_seq, int seq_len, float* __restrict__ conf,
                  int32_t* __restrict__ pred) {
+  pdl_prologue();
   const int n = *n_rows, lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
   for (int r = blockIdx.x * wpb + (threadIdx.x >> 5); r < n; r += gridDim.x * wpb) {
@@ -46,9 +47,7 @@ int launch_lm_reduce(const float* st_max, const float* st_sum, const int32_t* st
                      const int32_t* row_seq, int seq_len, float* conf, int32_t* pred, cudaStream_t st) {
   if (max_rows <= 0) return D2C_OK;
   const int grid = ceil_div(max_rows, 4) < 148 * 4 ? ceil_div(max_rows, 4) : 148 * 4;
-  lm_reduce_kernel<<<grid, 128, 0, st>>>(st_max, st_sum, st_arg, n_tiles, n_rows, lm_rows, sel_idx, row_seq,
-                                         seq_len, conf, pred);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((lm_reduce_kernel), grid, 128, 0, st, st_max, st_sum, st_arg, n_tiles, n_rows, lm_rows, sel_idx, row_seq, seq_len, conf, pred);
   return D2C_OK;
 }
 

@@ -12,6 +12,7 @@ namespace d2c {
 namespace {
 
 __global__ void rollout_init_kernel(RolloutArgs a, uint8_t* insel) {
+  pdl_prologue();
   const int b = blockIdx.y, L = a.seq_len;
   const int ro = a.row_off[b], nb = a.row_off[b + 1] - ro;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < L; j += gridDim.x * blockDim.x) {
@@ -30,6 +31,7 @@ __global__ void rollout_init_kernel(RolloutArgs a, uint8_t* insel) {
 
 __global__ void __launch_bounds__(256)
 rollout_partial_kernel(RolloutArgs a, const float* __restrict__ abar_l, const float* __restrict__ u) {
+  pdl_prologue();
   const int b = blockIdx.z, s = blockIdx.y, L = a.seq_len;
   const int j = blockIdx.x * 256 + threadIdx.x;
   const int ro = a.row_off[b], nb = a.row_off[b + 1] - ro;
@@ -50,6 +52,7 @@ rollout_partial_kernel(RolloutArgs a, const float* __restrict__ abar_l, const fl
 __global__ void __launch_bounds__(256)
 rollout_combine_kernel(RolloutArgs a, const uint8_t* __restrict__ insel, const float* __restrict__ u,
                        float* __restrict__ out) {
+  pdl_prologue();
   const int b = blockIdx.y, L = a.seq_len;
   const int j = blockIdx.x * 256 + threadIdx.x;
   if (j >= L || a.row_off[b + 1] - a.row_off[b] <= 0) return;
@@ -64,16 +67,13 @@ int launch_rollout(const RolloutArgs& a, cudaStream_t st) {
   if (a.batch <= 0 || a.seq_len <= 0 || a.n_layers <= 0) return D2C_OK;
   const int L = a.seq_len;
   uint8_t* insel = reinterpret_cast<uint8_t*>(a.partial + (size_t)a.n_split * a.batch * L);
-  rollout_init_kernel<<<dim3(ceil_div(L, 256), a.batch), 256, 0, st>>>(a, insel);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((rollout_init_kernel), dim3(ceil_div(L, 256), a.batch), 256, 0, st, a, insel);
   const float* u = a.u0;
   float* bufs[2] = {a.u1, a.u0};
   for (int l = a.n_layers - 1; l >= 0; --l) {
     float* out = (l == 0) ? a.c : bufs[(a.n_layers - 1 - l) & 1];
-    rollout_partial_kernel<<<dim3(ceil_div(L, 256), a.n_split, a.batch), 256, 0, st>>>(a, a.abar + (size_t)l * a.layer_stride, u);
-    D2C_LAUNCHED();
-    rollout_combine_kernel<<<dim3(ceil_div(L, 256), a.batch), 256, 0, st>>>(a, insel, u, out);
-    D2C_LAUNCHED();
+    D2C_LAUNCH((rollout_partial_kernel), dim3(ceil_div(L, 256), a.n_split, a.batch), 256, 0, st, a, a.abar + (size_t)l * a.layer_stride, u);
+    D2C_LAUNCH((rollout_combine_kernel), dim3(ceil_div(L, 256), a.batch), 256, 0, st, a, insel, u, out);
     u = out;
   }
   return D2C_OK;

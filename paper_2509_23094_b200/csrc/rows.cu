@@ -29,6 +29,7 @@ norm_rows_kernel(const bf16* __restrict__ src, const int32_t* __restrict__ sel_i
                  const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_map,
                  const int32_t* __restrict__ n_rows, int seq_len, int d, const bf16* __restrict__ gain,
                  float eps, bf16* __restrict__ x, bf16* __restrict__ xn) {
+  pdl_prologue();
   __shared__ float sh[kRowThreads / 32];
   const int n = *n_rows;
   for (int r = blockIdx.x; r < n; r += gridDim.x) {
@@ -67,18 +68,14 @@ int launch_gather_norm(const bf16* h0, const int32_t* sel_idx, const int32_t* ro
                        int max_rows, int seq_len, int d, const bf16* gain, float eps, bf16* x, bf16* xn,
                        cudaStream_t st) {
   if (max_rows <= 0) return D2C_OK;
-  norm_rows_kernel<true><<<row_grid(max_rows), kRowThreads, 0, st>>>(h0, sel_idx, row_seq, nullptr, n_rows,
-                                                                      seq_len, d, gain, eps, x, xn);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((norm_rows_kernel<true>), row_grid(max_rows), kRowThreads, 0, st, h0, sel_idx, row_seq, nullptr, n_rows, seq_len, d, gain, eps, x, xn);
   return D2C_OK;
 }
 
 int launch_rmsnorm(const bf16* x, const int32_t* row_map, const int32_t* n_rows, int max_rows, int d,
                    const bf16* gain, float eps, bf16* xn, cudaStream_t st) {
   if (max_rows <= 0) return D2C_OK;
-  norm_rows_kernel<false><<<row_grid(max_rows), kRowThreads, 0, st>>>(x, nullptr, nullptr, row_map, n_rows, 0, d,
-                                                                       gain, eps, nullptr, xn);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((norm_rows_kernel<false>), row_grid(max_rows), kRowThreads, 0, st, x, nullptr, nullptr, row_map, n_rows, 0, d, gain, eps, nullptr, xn);
   return D2C_OK;
 }
 
@@ -108,6 +105,7 @@ rope_scatter_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ sel_idx,
                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ n_rows, int hq, int hkv,
                     int dh, const float2* __restrict__ rope, bf16* __restrict__ kc, bf16* __restrict__ vc,
                     int cache_seq) {
+  pdl_prologue();
   const int n = *n_rows;
   const int half = dh >> 1, chunks = half >> 3;            // 16-byte chunks per half head
   const int ld = (hq + 2 * hkv) * dh;
@@ -145,9 +143,7 @@ int launch_rope_scatter(bf16* qkv, const int32_t* sel_idx, const int32_t* row_se
                         int max_rows, int hq, int hkv, int dh, const float2* rope, bf16* kc, bf16* vc,
                         int cache_seq, cudaStream_t st) {
   if (max_rows <= 0) return D2C_OK;
-  rope_scatter_kernel<<<row_grid(max_rows), kRowThreads, 0, st>>>(qkv, sel_idx, row_seq, n_rows, hq, hkv, dh, rope,
-                                                                   kc, vc, cache_seq);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((rope_scatter_kernel), row_grid(max_rows), kRowThreads, 0, st, qkv, sel_idx, row_seq, n_rows, hq, hkv, dh, rope, kc, vc, cache_seq);
   return D2C_OK;
 }
 

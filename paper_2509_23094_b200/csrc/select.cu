@@ -66,6 +66,7 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* warp_buf, T* total) {
 __device__ __forceinline__ float clean_score(float x) { return (x > 0.f && x < INFINITY) ? fminf(x, 262144.f) : 0.f; }
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P2) {
+  pdl_prologue();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t* sbuf = reinterpret_cast<uint64_t*>(smem_raw);
   uint8_t* flags = reinterpret_cast<uint8_t*>(sbuf + P2);
@@ -212,6 +213,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
 
 // Turns the per-sequence ranks into global row numbers.
 __global__ void __launch_bounds__(256) select_finalize_kernel(SelectArgs a) {
+  pdl_prologue();
   const int b = blockIdx.y, L = a.seq_len;
   int off = 0, lmoff = 0;
   for (int bb = 0; bb < b; ++bb) { off += a.n_b[bb]; lmoff += a.nm_b[bb]; }
@@ -245,11 +247,9 @@ int launch_select(const SelectArgs& a, cudaStream_t st) {
     D2C_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8192 * 8 + 2 * 8192));
     attr_set = true;
   }
-  select_kernel<<<a.batch, kSelThreads, smem, st>>>(a, P2);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((select_kernel), a.batch, kSelThreads, smem, st, a, P2);
   dim3 grid(ceil_div(a.seq_len, 256), a.batch);
-  select_finalize_kernel<<<grid, 256, 0, st>>>(a);
-  D2C_LAUNCHED();
+  D2C_LAUNCH((select_finalize_kernel), grid, 256, 0, st, a);
   return D2C_OK;
 }
 
