@@ -45,50 +45,62 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons through NVML (read-only queries) from a thread while the
+    timed region runs; nvidia-smi's own sampling period is longer than a whole timed pass of the small
+    workloads.  Falls back to one nvidia-smi query if NVML cannot be loaded."""
 
     def __init__(self, index: int):
-        self.index, self.proc, self.file = index, None, None
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop, self._thread, self._nvml = False, None, None
+
+    def _loop(self):
+        nv, h = self._nvml, self._handle
+        bits = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown, "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown, "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+        while not self._stop:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                for name, bit in bits.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
         try:
-            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=self.file, stderr=subprocess.DEVNULL)
+            import pynvml as nv
+            nv.nvmlInit()
+            # NVML counts physical devices; honour CUDA_VISIBLE_DEVICES when it lists ordinals
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            ids = [v for v in vis.split(",") if v.strip().isdigit()]
+            phys = int(ids[self.index]) if self.index < len(ids) else self.index
+            self._handle = nv.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(self._handle, nv.NVML_CLOCK_SM))
+            self._nvml = nv
+            import threading
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
         except Exception:
-            self.proc = None
+            self._nvml = None
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
+        if self._nvml is not None:
+            self._stop = True
+            self._thread.join(timeout=2)
+            if self.samples:
+                out.update(sm_mhz=float(statistics.median(self.samples)), sm_max_mhz=self.max_mhz,
+                           reasons=sorted(self.reasons), samples=len(self.samples))
             return out
-        self.proc.terminate()
         try:
-            self.proc.wait(timeout=5)
+            q = "clocks.sm,clocks.max.sm"
+            txt = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}", "--format=csv,noheader,nounits"],
+                                 capture_output=True, text=True, timeout=10).stdout.strip().split(",")
+            out.update(sm_mhz=float(txt[0]), sm_max_mhz=float(txt[1]), samples=1)
         except Exception:
-            self.proc.kill()
-        self.file.flush()
-        self.file.seek(0)
-        clocks, reasons, mx = [], set(), None
-        for line in self.file:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 8:
-                continue
-            try:
-                clocks.append(float(parts[0])); mx = float(parts[1])
-            except ValueError:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        self.file.close()
-        os.unlink(self.file.name)
-        if clocks:
-            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks))
+            pass
         return out
 
 
@@ -140,7 +152,6 @@ def run_ours(args, rank, world, device):
     ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     sampler = ClockSampler(torch.cuda.current_device())
-    sampler.start()                      # sampled from the warm-up on: the timed passes alone can be shorter than one sample
     for _ in range(args.warmup):
         restore()
         ctx.step(h0, mask_dev, wl.k, wl.p, hidden_out=hid)
@@ -175,6 +186,7 @@ def run_ours(args, rank, world, device):
     # Pass 1 gives the headline: no events inside the step, so the kernels' programmatic dependent
     # launches overlap as they do for a user.  Pass 2 repeats the same K steps with one event at every
     # phase boundary (which serialises the launches) and gives the per-phase and per-kernel times.
+    sampler.start()
     per_step_ms, _ = timed_pass(False)
     per_step_ms_profiled, phases = timed_pass(True)
     clocks = sampler.stop()
@@ -248,9 +260,41 @@ def run_ours(args, rank, world, device):
         "step_ms_min": round(min(per_step_ms), 4), "step_ms_median": round(statistics.median(per_step_ms), 4),
         "ms_per_step_with_phase_events": round(sum(per_step_ms_profiled) / args.steps, 4),
     }
+    if args.decode:
+        line["decode"] = decode_loop(ctx, wl, w_dev, mask, tokens, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L)
     return line
+
+
+def decode_loop(ctx, wl, w_dev, mask, tokens, device):
+    """The whole decoding loop of the workload (Eq. 2): prefill, then until no [MASK] is left: commit
+    the most confident refreshed position of every sequence, run one d2c_step with that position forced.
+    Everything stays on the device; the host synchronises once at the end."""
+    B, L = wl.batch, wl.seq_len
+    gen = int(mask[0].sum())
+    mask_dev = mask.to(device).contiguous()
+    tok = tokens.to(torch.int32).to(device).contiguous()
+    h0 = w_dev["embed"][tokens.to(device)].contiguous()
+    committed = torch.full((B,), -1, dtype=torch.int32, device=device)
+    forced_off = torch.arange(B + 1, dtype=torch.int32, device=device)
+    torch.cuda.synchronize()
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    stream = torch.cuda.current_stream()
+    e0.record(stream)
+    ctx.step(h0, mask_dev, 10 ** 6, 1.0)
+    e1.record(stream)
+    for _ in range(gen):
+        ctx.commit(w_dev["embed"], h0, mask_dev, tok, committed, rule=0)
+        ctx.step(h0, mask_dev, wl.k, wl.p, forced=committed, forced_off=forced_off)
+    e2.record(stream)
+    torch.cuda.synchronize()
+    ctx.sync_status()
+    left = int(mask_dev.sum())
+    prefill_ms, loop_ms = e0.elapsed_time(e1), e1.elapsed_time(e2)
+    return {"generated_tokens": B * gen - left, "masks_left": left, "steps": gen, "prefill_ms": round(prefill_ms, 3),
+            "ms_per_step": round(loop_ms / gen, 4), "tokens_per_s": round((B * gen - left) / ((prefill_ms + loop_ms) * 1e-3), 2),
+            "total_s": round((prefill_ms + loop_ms) * 1e-3, 4)}
 
 
 def oracle_setup(wl, w_cpu, mask, tokens):
@@ -339,6 +383,7 @@ def main():
     ap.add_argument("--workload", default="llada1l_1024", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode", action="store_true", help="also run the workload's whole decoding loop")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

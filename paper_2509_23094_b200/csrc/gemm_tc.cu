@@ -131,13 +131,19 @@ template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant__ CUtensorMap tmA64,
                const __grid_constant__ CUtensorMap tmA32, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmB64, const TcParams p) {
   pdl_prologue();
-  constexpr int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : 256;  // output columns per tile
   const GemmArgs& g = p.g;
   const int n = *g.n_rows;
   if (n <= 0) return;
-  const int MT = (n + TM - 1) / TM, NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int MT = (n + TM - 1) / TM;
+  // Accumulator width of this launch: 256 columns, narrowed to 128 or 64 while that still leaves SMs
+  // without a tile (few live rows and a small N), so that more SMs stream the weights.
+  int bn = ACC_COLS;
+  const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : 64);
+  while (bn > bn_min && 2 * MT * ((g.N + bn - 1) / bn) <= (int)gridDim.x) bn >>= 1;
+  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
+  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
   const int total = MT * NT;
   if ((int)blockIdx.x >= total) return;                      // uniform: nothing allocated yet
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -186,11 +192,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
           const int s = it % ST;
           if (!mbar_wait(empty_bar(s), ((it / ST) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(s), a_bytes + B_BYTES);
+          mbar_expect_tx(full_bar(s), a_bytes + (uint32_t)bn * TK * 2);
           tma_load_2d(sa, ma, kt * TK, m0, full_bar(s));
-          tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
-          if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
-          else tma_load_2d(sb + 128 * TK * 2, &tmB, kt * TK, n0 + 128, full_bar(s));
+          if (bn == 64) {
+            tma_load_2d(sb, &tmB64, kt * TK, n0, full_bar(s));
+          } else {
+            tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
+            if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
+            else if (bn == 256) tma_load_2d(sb + 128 * TK * 2, &tmB, kt * TK, n0 + 128, full_bar(s));
+          }
         }
       }
       if (*abortp) {
@@ -205,7 +215,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(ACC_COLS);
+      const uint32_t idesc = instr_desc(bn);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++tcount) {
@@ -236,6 +246,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tcount) {
       const uint32_t buf = tcount & 1, use = tcount >> 1;
       const int m0 = (tile % MT) * TM, nt = tile / MT, n0 = nt * OUT_COLS;
+      const int n_chunks = OUT_COLS / 32;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 3)) break;
@@ -244,7 +255,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
-        for (int c = 0; c < OUT_COLS / 32; ++c) {
+        for (int c = 0; c < n_chunks; ++c) {
           uint32_t v[32];
           tmem_ld32(tbase + c * 32, v);
           tmem_ld_wait();
@@ -283,7 +294,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         }
       } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-        for (int c = 0; c < OUT_COLS / 32; ++c) {
+        for (int c = 0; c < n_chunks; ++c) {
           uint32_t gv[32], uv[32];
           tmem_ld32(tbase + c * 32, gv);
           tmem_ld32(tbase + 128 + c * 32, uv);
@@ -315,7 +326,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         }
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
-        for (int half = 0; half < 2; ++half) {                // statistics are kept per 128 columns
+        for (int half = 0; half < bn / 128; ++half) {         // statistics are kept per 128 columns
           float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
@@ -345,7 +356,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
                 if (col0 + j < g.N) lp[j] = __uint_as_float(v[j]);
             }
           }
-          const int stile = nt * 2 + half;
+          const int stile = nt * (bn / 128) + half;
           if (row_ok && stile < g.n_tiles) {
             const size_t o = (size_t)row * g.n_tiles + stile;
             g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
@@ -417,18 +428,19 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_set = true;
   }
-  CUtensorMap tmA128, tmA64, tmA32, tmB, tmB2;
+  CUtensorMap tmA128, tmA64, tmA32, tmB, tmB2, tmB64;
   int rc = make_map(&tmA128, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
   if (rc == D2C_OK) rc = make_map(&tmA64, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 64);
   if (rc == D2C_OK) rc = make_map(&tmA32, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 32);
   if (rc == D2C_OK) rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
   if (rc == D2C_OK) rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
+  if (rc == D2C_OK) rc = make_map(&tmB64, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 64);
   if (rc != D2C_OK) return rc;
   TcParams p{g, status};
-  const int out_cols = EPI == EPI_SWIGLU ? 128 : 256;
+  const int out_cols = EPI == EPI_SWIGLU ? 128 : (EPI == EPI_LMSTATS ? 128 : 64);   // narrowest tile the kernel may pick
   const long long tiles = (long long)ceil_div(g.max_rows, TM) * ceil_div(g.N, out_cols);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  D2C_LAUNCH((gemm_tc_kernel<EPI>), grid, TC_THREADS, smem, st, tmA128, tmA64, tmA32, tmB, tmB2, p);
+  D2C_LAUNCH((gemm_tc_kernel<EPI>), grid, TC_THREADS, smem, st, tmA128, tmA64, tmA32, tmB, tmB2, tmB64, p);
   return D2C_OK;
 }
 }  // namespace

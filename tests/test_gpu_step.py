@@ -161,3 +161,48 @@ def test_step_host_matches_device_step():
     np.testing.assert_array_equal(sel.numpy()[:n], np.concatenate(g["sel"]))
     np.testing.assert_array_equal(hid.float().numpy()[:n], np.concatenate(g["hidden"]))
     assert torch.equal(conf, conf_dev)
+
+
+@pytest.mark.parametrize("rule", [0, 1, 2])
+def test_decode_loop_commits_match_the_oracle_rule(rule):
+    """commit + step for several iterations: every commit decision is checked against the oracle's
+    scheduling function applied to the confidences the GPU holds, every step's selection against the
+    oracle's selection, and the final hidden states against a teacher-forced oracle."""
+    from oracle import decode
+    wl = WLS["gqa_bias_3layers"]
+    pair = Pair(wl)
+    _prefill(pair)
+    B, L = wl.batch, wl.seq_len
+    mask = pair.mask.clone().cuda(); h0 = pair.h0.clone().cuda()
+    tokens = pair.tokens.to(torch.int32).cuda().contiguous()
+    committed = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    embed = pair.w_dev["embed"]
+    fresh = [np.flatnonzero(pair.mask[b].numpy()) for b in range(B)]              # the prefill refreshed every masked row
+    for it in range(5):
+        conf = pair.ctx.view("conf", B, L).cpu().numpy(); pred = pair.ctx.view("pred", B, L).cpu().numpy()
+        mask_before = mask.cpu().numpy()
+        pair.ctx.commit(embed, h0, mask, tokens, committed, rule=rule, threshold=0.002)
+        torch.cuda.synchronize()
+        got_mask = mask.cpu().numpy(); forced = []
+        for b in range(B):
+            want, best = decode.commit(mask_before[b], conf[b], fresh[b], rule=rule, sigma=wl.sigma, threshold=0.002)
+            assert int(committed[b]) == best
+            assert np.flatnonzero(mask_before[b] != got_mask[b]).tolist() == want
+            for pos in want:
+                assert int(tokens[b, pos]) == int(pred[b, pos]) and torch.equal(h0[b, pos], embed[int(pred[b, pos])])
+            forced.append(want[:1] if rule != 2 else want)
+        f = torch.tensor([x for fb in forced for x in fb] or [0], dtype=torch.int32, device="cuda")
+        fo = torch.tensor(np.cumsum([0] + [len(fb) for fb in forced]), dtype=torch.int32, device="cuda")
+        conf_b = pair.ctx.view("conf", B, L).cpu().numpy().copy(); c_b = pair.ctx.view("c", B, L).cpu().numpy().copy()
+        hid = torch.zeros(B * L, wl.shape.d_model, dtype=torch.bfloat16, device="cuda")
+        pair.ctx.step(h0, mask, wl.k, 0.3, forced=f, forced_off=fo, hidden_out=hid)
+        pair.ctx.sync_status()
+        ro = pair.ctx.view("row_off", B, L).cpu().numpy(); sel = pair.ctx.view("sel_idx").cpu().numpy()
+        S = [sel[ro[b]: ro[b + 1]].astype(np.int64) for b in range(B)]
+        want_sel = pair.oracle_selection(conf_b, c_b, mask.cpu(), wl.k, 0.3, forced=forced)
+        for b in range(B):
+            np.testing.assert_array_equal(S[b], want_sel[b])
+        res = pair.oracle_step(S, mask=mask.cpu(), h0=h0.cpu())
+        for b in range(B):
+            assert row_rel_err(hid[ro[b]: ro[b + 1]].float().cpu().numpy(), res.hidden[b]) <= ROW_TOL
+        fresh = [np.array([p for p in S[b] if got_mask[b, p]]) for b in range(B)]

@@ -100,3 +100,18 @@ def test_repeated_select_all_steps_are_idempotent():
     b = ostep.oracle_step(st, wf, shape, h, mask, k=10 ** 6, p=1.0)
     np.testing.assert_allclose(a.hidden[0], b.hidden[0], atol=1e-13)
     np.testing.assert_array_equal(c1, st.c)
+
+
+def test_commit_rules():
+    from oracle import decode
+    mask = np.zeros(200, dtype=np.uint8); mask[100:] = 1
+    conf = np.zeros(200, dtype=np.float32)
+    conf[[100, 120, 150]] = [0.5, 0.9, 0.95]
+    elig = [100, 120, 150, 160]
+    assert decode.commit(mask, conf, elig, rule=0) == ([150], 150)                # highest confidence
+    assert decode.commit(mask, conf, elig, rule=1) == ([100], 100)                # next to the known prefix wins
+    assert decode.commit(mask, conf, elig, rule=2, threshold=0.8) == ([120, 150], 150)
+    assert decode.commit(mask, conf, elig, rule=2, threshold=0.99) == ([150], 150)
+    assert decode.commit(mask, conf, [5, 7], rule=0) == ([], -1)                   # known positions are not eligible
+    conf[[120, 150]] = 0.9
+    assert decode.commit(mask, conf, elig, rule=0) == ([120], 120)                # tie: lower position
