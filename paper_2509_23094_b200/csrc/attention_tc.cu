@@ -123,7 +123,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-struct AttnTcParams { AttnArgs a; int* status; };
+struct AttnTcParams { AttnArgs a; int* status; int sm_count; int head_groups; };
 
 // ------------------------------------------------------------------------------------------------
 // Forward kernel.  One CTA owns up to 256 selected rows of one (sequence, head): two query tiles of
@@ -150,8 +150,12 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   pdl_prologue();
   const AttnArgs& a = p.a;
   const int b = blockIdx.z, h = blockIdx.y, g = h / (a.hq / a.hkv);
-  const int r0 = a.row_off[b] + blockIdx.x * 2 * AQ;
-  const int nrows = min(2 * AQ, a.row_off[b + 1] - r0);
+  // With few selected rows every 128-row tile gets a CTA of its own (more SMs busy); otherwise a CTA
+  // takes two tiles, which halves the K/V traffic per row and keeps both softmax warp groups busy.
+  const int nb = a.row_off[b + 1] - a.row_off[b];
+  const bool pairs = ((nb + AQ - 1) / AQ) * a.hq * a.batch > p.sm_count;
+  const int r0 = a.row_off[b] + blockIdx.x * (pairs ? 2 * AQ : AQ);
+  const int nrows = min(pairs ? 2 * AQ : AQ, a.row_off[b + 1] - r0);
   if (nrows <= 0) return;                                          // uniform: nothing allocated yet
   const int nq = nrows > AQ ? 2 : 1;                                // live query tiles
   const int L = a.seq_len, T = (L + AKEYS - 1) / AKEYS;
@@ -366,10 +370,12 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const int b = blockIdx.z;
   const int r0 = a.row_off[b] + blockIdx.y * AQ;
   const int nrows = min(AQ, a.row_off[b + 1] - r0);
-  const int key0 = blockIdx.x * AKEYS, L = a.seq_len;
-  if (nrows <= 0 || key0 >= L) return;
+  const int L = a.seq_len, ktiles = (L + AKEYS - 1) / AKEYS;
+  const int key0 = ((int)blockIdx.x % ktiles) * AKEYS, hg = (int)blockIdx.x / ktiles;
+  if (nrows <= 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = a.hq / a.hkv;
+  const int nh = a.hq / p.head_groups, h_first = hg * nh;          // this CTA's heads (whole kv groups)
   int* status = p.status ? p.status : g_attn_status;
 
   extern __shared__ unsigned char smem_raw[];
@@ -405,18 +411,18 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   if (warp == 0) {
     if (lane == 0) {
       int issued = 0;
-      for (int h = 0; h < a.hq; ++h) {
-        const int s = h % ABS, u = h / ABS;
+      for (int h = 0; h < nh; ++h) {                                // h: local head index, hgl: head of the model
+        const int s = h % ABS, u = h / ABS, hgl = h_first + h;
         if (!mbar_wait(QE(s), (u & 1) ^ 1, abortp, status, 21)) break;
         mbar_expect_tx(QF(s), TILE_BYTES);
-        tma_load_2d(sQ(s), &tmQ, h * ADH, r0, QF(s));
-        tma_load_2d(sQ(s) + HALF_BYTES, &tmQ, h * ADH + 64, r0, QF(s));
+        tma_load_2d(sQ(s), &tmQ, hgl * ADH, r0, QF(s));
+        tma_load_2d(sQ(s) + HALF_BYTES, &tmQ, hgl * ADH + 64, r0, QF(s));
         if (h % group == 0) {
-          const int gi = h / group, ks = gi % ABS, ku = gi / ABS;
+          const int gi = h / group, ks = gi % ABS, ku = gi / ABS, ggl = hgl / group;
           if (!mbar_wait(KE(ks), (ku & 1) ^ 1, abortp, status, 22)) break;
           mbar_expect_tx(KF(ks), TILE_BYTES);
-          tma_load_2d(sK(ks), &tmK, gi * ADH, kv_row, KF(ks));
-          tma_load_2d(sK(ks) + HALF_BYTES, &tmK, gi * ADH + 64, kv_row, KF(ks));
+          tma_load_2d(sK(ks), &tmK, ggl * ADH, kv_row, KF(ks));
+          tma_load_2d(sK(ks) + HALF_BYTES, &tmK, ggl * ADH + 64, kv_row, KF(ks));
         }
         issued = h + 1;
       }
@@ -430,7 +436,7 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
-      for (int h = 0; h < a.hq; ++h) {
+      for (int h = 0; h < nh; ++h) {
         const int s = h % ABS, u = h / ABS, gi = h / group, ks = gi % ABS, ku = gi / ABS, sb = h & 1;
         if (!mbar_wait(QF(s), u & 1, abortp, status, 23)) break;
         if (h % group == 0 && !mbar_wait(KF(ks), ku & 1, abortp, status, 24)) break;
@@ -442,7 +448,7 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           umma_ss(tm + sb * 128, desc_kmajor(sQ(s) + off) + 2 * (i & 3), desc_kmajor(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
         }
         umma_commit(QE(s));                                         // Q stage free
-        if ((h + 1) % group == 0 || h + 1 == a.hq) umma_commit(KE(ks));      // last head of the group: K stage free
+        if ((h + 1) % group == 0 || h + 1 == nh) umma_commit(KE(ks));        // last head of the group: K stage free
         umma_commit(SF(sb));
       }
     }
@@ -458,9 +464,9 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
     for (int i = 0; i < 64; ++i) acc[i] = 0.f;
     bool ok = true;
-    for (int h = 0; h < a.hq && ok; ++h) {
+    for (int h = 0; h < nh && ok; ++h) {
       const int sb = h & 1;
-      const float e = row_ok ? a.lse[(size_t)(r0 + lrow) * a.hq + h] * kLog2e : 0.f;
+      const float e = row_ok ? a.lse[(size_t)(r0 + lrow) * a.hq + h_first + h] * kLog2e : 0.f;
       if (!mbar_wait(SF(sb), (h >> 1) & 1, abortp, status, 26)) { ok = false; break; }
       tc_fence_after();
       uint32_t v[2][32];
@@ -478,7 +484,8 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (ok && row_ok) {
       const float inv = 1.f / (float)a.hq;
       const int k0 = key0 + half * 64;
-      float* dst = a.abar + (size_t)(r0 + lrow) * L + k0;
+      float* out = p.head_groups > 1 ? a.abar_partial + (size_t)hg * ((size_t)a.q_rows * L) : a.abar;
+      float* dst = out + (size_t)(r0 + lrow) * L + k0;
       if (k0 + 64 <= L && (L & 3) == 0) {
 #pragma unroll
         for (int q = 0; q < 16; ++q)
@@ -493,6 +500,24 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   tc_fence_before();
   __syncthreads();
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tm, 256); }
+}
+
+// Abar = sum of the head groups' partial sums, in group order (deterministic).
+__global__ void __launch_bounds__(256)
+abar_sum_kernel(const float* __restrict__ part, size_t group_stride, int groups, const int32_t* __restrict__ n_rows,
+                int L, float* __restrict__ abar) {
+  pdl_prologue();
+  const size_t total4 = ((size_t)(*n_rows) * L) >> 2;               // L is a multiple of 4 on this path
+  const float4* p4 = reinterpret_cast<const float4*>(part);
+  const size_t gs4 = group_stride >> 2;
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < total4; i += (size_t)gridDim.x * 256) {
+    float4 acc = p4[i];
+    for (int g2 = 1; g2 < groups; ++g2) {
+      const float4 t = p4[i + (size_t)g2 * gs4];
+      acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    }
+    reinterpret_cast<float4*>(abar)[i] = acc;
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -546,13 +571,25 @@ int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   if (rc == D2C_OK) rc = make_map(&tmK, a.kc, kv_rows, kv_cols, kv_cols);
   if (rc == D2C_OK) rc = make_map(&tmV, a.vc, kv_rows, kv_cols, kv_cols);
   if (rc != D2C_OK) return rc;
-  AttnTcParams p{a, status};
-  const int qtiles = ceil_div(a.max_rows_per_seq, AQ);
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 148;
+  const int qtiles = ceil_div(a.max_rows_per_seq, AQ), ktiles = ceil_div(a.seq_len, AKEYS);
+  // split the heads over several CTAs while the (row tile x key tile) grid leaves a quarter of the SMs idle
+  int groups = 1;
+  const int kv_group = a.hq / a.hkv;
+  while (a.abar_partial && a.n_rows && (a.seq_len & 3) == 0 && groups < 8 && 4LL * ktiles * qtiles * a.batch * groups < 3LL * sms &&
+         a.hq % (groups * 2) == 0 && (a.hq / (groups * 2)) % kv_group == 0 &&
+         (size_t)(groups * 2) * a.q_rows * a.seq_len <= a.abar_partial_floats)
+    groups *= 2;
+  AttnTcParams p{a, status, sms, groups};
   if (a.which != 2) {
-    D2C_LAUNCH((attn_fwd_tc), dim3(ceil_div(a.max_rows_per_seq, 2 * AQ), a.hq, a.batch), FWD_THREADS, smem_fwd, st, tmQ, tmK, tmV, p);
+    D2C_LAUNCH((attn_fwd_tc), dim3(qtiles, a.hq, a.batch), FWD_THREADS, smem_fwd, st, tmQ, tmK, tmV, p);
   }
   if (a.abar && a.which != 1) {
-    D2C_LAUNCH((attn_abar_tc), dim3(ceil_div(a.seq_len, AKEYS), qtiles, a.batch), FWD_THREADS, smem_ab, st, tmQ, tmK, p);
+    D2C_LAUNCH((attn_abar_tc), dim3(ktiles * groups, qtiles, a.batch), FWD_THREADS, smem_ab, st, tmQ, tmK, p);
+    if (groups > 1)
+      D2C_LAUNCH((abar_sum_kernel), 4 * sms, 256, 0, st, (const float*)a.abar_partial, (size_t)a.q_rows * a.seq_len, groups, a.n_rows,
+                 a.seq_len, a.abar);
   }
   return D2C_OK;
 }

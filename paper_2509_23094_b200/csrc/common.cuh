@@ -105,6 +105,9 @@ struct AttnArgs {
   int portable;                          // 1: force the mma.sync kernels
   int* status;                           // device status word for bounded waits (may be null)
   int which;                             // 0: both kernels, 1: O/LSE only, 2: head-averaged probabilities only
+  // optional scratch that lets the abar kernel split the heads over several CTAs when the problem has too few
+  // (rows x keys) tiles to fill the GPU: partial sums [head group][rows][seq_len], added in a fixed order
+  float* abar_partial; size_t abar_partial_floats; const int32_t* n_rows;
 };
 int launch_attention(const AttnArgs& a, cudaStream_t st);
 bool attention_tc_supported(const AttnArgs& a);               // attention_tc.cu

@@ -44,6 +44,7 @@ struct Buffers {
   bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar;
   float *st_max, *st_sum; int32_t* st_arg;
   float *u0, *u1, *partial;
+  float* abar_part; size_t abar_part_floats;
   bf16* h0_stage; uint8_t* mask_stage; int32_t *forced_stage, *forced_off_stage; float *okey_stage, *oc_stage;
   int32_t* committed_stage;
 };
@@ -74,6 +75,10 @@ static size_t carve(const d2c_config& c, void* base, Buffers* out) {
   b.st_max = w.take<float>(R * nt); b.st_sum = w.take<float>(R * nt); b.st_arg = w.take<int32_t>(R * nt);
   b.u0 = w.take<float>(R); b.u1 = w.take<float>(R);
   b.partial = w.take<float>((size_t)kRolloutSplit * R + (R + 3) / 4);     // partial sums + selected-flag bytes
+  // scratch for the head-split of the abar kernel: only worth having when the (rows x keys) grid is small
+  const size_t tiles_worst = (size_t)ceil_div((int)L, 128) * ceil_div((int)L, 128) * B;
+  b.abar_part_floats = tiles_worst < 2 * 160 ? (size_t)8 * R * L : 0;
+  b.abar_part = w.take<float>(b.abar_part_floats);
   b.h0_stage = w.take<bf16>(R * d); b.mask_stage = w.take<uint8_t>(R);
   b.forced_stage = w.take<int32_t>(R); b.forced_off_stage = w.take<int32_t>(B + 1);
   b.okey_stage = w.take<float>(R); b.oc_stage = w.take<float>(R); b.committed_stage = w.take<int32_t>(B);
@@ -297,6 +302,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     at.q = b.qkv; at.ldq = qkv_out; at.kc = kc; at.vc = vc; at.row_off = b.row_off; at.batch = B; at.seq_len = L;
     at.cache_seq = c.max_seq; at.hq = hq; at.hkv = hkv; at.dh = dh; at.max_rows_per_seq = L;
     at.q_rows = R; at.portable = (c.flags & D2C_FLAG_PORTABLE_ATTENTION) ? 1 : 0; at.status = b.status;
+    at.abar_partial = b.abar_part_floats ? b.abar_part : nullptr; at.abar_partial_floats = b.abar_part_floats; at.n_rows = n_rows;
     at.o = b.o; at.lse = b.lse; at.abar = l < depth ? b.abar + (size_t)l * c.max_batch * c.max_seq * c.max_seq : nullptr;
     D2C_TRY(ctx, mark(ctx, PH_ATTN));
     at.which = 1;

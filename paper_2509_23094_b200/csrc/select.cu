@@ -86,6 +86,87 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
   if (tid == 0) { s_cnt = 0; }
   __syncthreads();
 
+  if (a.stage2_candidates == 0) {
+    // ---- default candidate mode: masked positions (stage 1) and known positions (stage 2) are disjoint,
+    //      so one sort orders both: bit 63 = masked, bits 62..32 = score bits, bits 31..0 = ~position ----
+    for (int i = tid; i < P2; i += kSelThreads) {
+      uint64_t comp = 0;
+      if (i < L) {
+        float key = 0.f;
+        if (smask[i]) {
+          if (okey) {
+            key = clean_score(okey[i]);
+          } else {
+            unsigned long long dq = 0;
+            for (int r = 1; r < a.phi_len; ++r) {
+              const int lo = i - r, hi = i + r;
+              int known = 0;
+              if (lo >= 0) known += 1 - smask[lo];
+              if (hi < L) known += 1 - smask[hi];
+              dq += (unsigned long long)a.phi_q30[r] * (unsigned)known;
+            }
+            const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;   // * 2^-30, exact
+            key = clean_score(__fmul_rn(D, conf[i]));
+          }
+          comp = (1ull << 63) | ((uint64_t)__float_as_uint(key) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
+        } else {
+          comp = ((uint64_t)__float_as_uint(clean_score(cs[i])) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
+        }
+        a.key[(size_t)b * L + i] = key;
+      }
+      sbuf[i] = comp;
+    }
+    bitonic_sort_desc(sbuf, P2);
+    if (tid == 0) { s_cnt = 0; s_take = 0; }                      // s_take doubles as the masked count here
+    __syncthreads();
+    for (int t = tid; t < P2; t += kSelThreads) {
+      const uint64_t x = sbuf[t], y = t + 1 < P2 ? sbuf[t + 1] : 0ull;
+      if ((x >> 63) && !(y >> 63)) s_take = t + 1;
+      if (x != 0 && y == 0) s_cnt = t + 1;
+    }
+    __syncthreads();
+    const int nm = s_take, ntot = s_cnt;
+    {
+      const int take = min(max(a.k, 0), nm);
+      for (int t = tid; t < take; t += kSelThreads) {
+        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
+        flags[idx] = F_SEL | F_MSTAR;
+      }
+    }
+    const int per = max(1, P2 / kSelThreads);
+    const int t0 = tid * per;
+    unsigned long long local = 0;
+    if (t0 < P2) {
+      for (int e = 0; e < per; ++e) {
+        const uint64_t x = sbuf[t0 + e];
+        if (!(x >> 63)) local += __double2ull_rd((double)__uint_as_float((uint32_t)(x >> 32)) * 4294967296.0);
+      }
+    }
+    const unsigned long long excl =
+        block_exclusive_scan<unsigned long long>(local, (unsigned long long*)warp_buf64, (unsigned long long*)&s_total64);
+    if (tid == 0) s_take = (a.p > 0.f) ? ntot : nm;                // end (exclusive) of the selected candidates
+    __syncthreads();
+    if (a.p > 0.f && t0 < P2) {
+      const double thr = __dmul_rn((double)a.p, __ull2double_rn(s_total64));
+      unsigned long long run = excl;
+      for (int e = 0; e < per; ++e) {
+        const int t = t0 + e;
+        if (t >= ntot) break;
+        if (t < nm) continue;
+        run += __double2ull_rd((double)__uint_as_float((uint32_t)(sbuf[t] >> 32)) * 4294967296.0);
+        if (__ull2double_rn(run) > thr) { atomicMin(&s_take, t + 1); break; }
+      }
+    }
+    __syncthreads();
+    {
+      const int end = s_take;
+      for (int t = nm + tid; t < end; t += kSelThreads) {
+        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
+        flags[idx] |= F_SEL;
+      }
+    }
+    __syncthreads();
+  } else {
   // ---- stage 1: keys ----
   for (int i = tid; i < P2; i += kSelThreads) {
     uint64_t comp = 0;
@@ -174,6 +255,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
     }
   }
   __syncthreads();
+
+  }
 
   // ---- forced rows ----
   if (a.forced && a.forced_off) {
