@@ -69,6 +69,7 @@ typedef struct {
 } d2c_config;
 #define D2C_FLAG_PORTABLE_GEMM 1        /* run the GEMMs on the mma.sync kernel instead of the tcgen05 one (cross-check) */
 #define D2C_FLAG_PORTABLE_ATTENTION 2   /* same for the attention kernels                                                */
+#define D2C_FLAG_ONE_SM_GEMM 4          /* keep the GEMMs on the one-SM tcgen05 kernel (no CTA pairs)                    */
 
 /* Weights.  The arrays of per-layer pointers are HOST arrays of n_layers DEVICE
  * pointers; they are copied at create, the device memory is borrowed for the
@@ -213,8 +214,9 @@ int d2c_op_select(const uint8_t* mask, const float* conf, const float* c, const 
 
 /* C[m][n] = sum_k A[m][k] * W[n][k] (+ bias[n]) in bf16 with fp32 accumulation,
  * for the first *n_rows rows (n_rows is a DEVICE int32, <= max_rows).  A: [max_rows][K],
- * W: [N][K], C: [max_rows][N].  K a multiple of 64.  impl 0: tcgen05/TMEM kernel,
- * impl 1: the portable mma.sync kernel. */
+ * W: [N][K], C: [max_rows][N].  K a multiple of 64.  impl 0: tcgen05/TMEM kernels (CTA pairs where
+ * the shape allows, else one SM per tile), impl 1: the portable mma.sync kernel, impl 2: the one-SM
+ * tcgen05 kernel. */
 int d2c_op_gemm(const void* A, const void* W, const void* bias, void* C, const int32_t* n_rows,
                 int32_t max_rows, int32_t N, int32_t K, int32_t impl, void* cuda_stream);
 

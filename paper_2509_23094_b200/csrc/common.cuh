@@ -136,4 +136,7 @@ int launch_commit(int batch, int seq_len, int d, int rule, float threshold, cons
 // ---- tcgen05 GEMM (gemm_tc.cu) -------------------------------------------------------------------
 // status: device int[4] that receives D2C_ETIMEOUT if a bounded wait runs out (null: a library-owned word).
 int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status = nullptr);
+// ---- two-SM tcgen05 GEMM (gemm_tc2.cu): pairs of CTAs on 256-row tiles ---------------------------
+bool gemm_tc2_supported(const GemmArgs& g);
+int launch_gemm_tc2(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status = nullptr);
 }  // namespace d2c

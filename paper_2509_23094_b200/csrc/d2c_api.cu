@@ -97,7 +97,7 @@ static const char* check_config(const d2c_config* c) {
   if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
   if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
   if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
-  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION))) return "rollout_layers >= 0 and no unknown flag bits required";
+  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION | D2C_FLAG_ONE_SM_GEMM))) return "rollout_layers >= 0 and no unknown flag bits required";
   return nullptr;
 }
 
@@ -155,6 +155,10 @@ static int pass(d2c_ctx* ctx, int rc) {
 // The step's GEMMs: tcgen05 kernel unless the context was created with D2C_FLAG_PORTABLE_GEMM.
 static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->stream);
+  // The LM head runs on few rows and is bound by the weight stream: the one-SM kernel sizes its A boxes to the
+  // live rows, a pair would load a second, empty row tile.
+  if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && gemm_tc2_supported(g))
+    return launch_gemm_tc2(g, epi, ctx->stream, ctx->buf.status);
   return launch_gemm_tc(g, epi, ctx->stream, ctx->buf.status);
 }
 #define D2C_TRY(ctx, expr) do { int rc__ = (expr); if (rc__ != D2C_OK) return pass((ctx), rc__); } while (0)

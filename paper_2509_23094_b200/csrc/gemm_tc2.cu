@@ -1,0 +1,478 @@
+// Two-SM tcgen05 GEMM (cta_group::2) with the same fused epilogues as gemm_tc.cu.
+//
+// A cluster of two CTAs (two SMs) computes a 256 x 256 accumulator tile: CTA r of the pair owns rows
+// [128 r, 128 r + 128) of the tile (its own TMEM holds them) and brings in only half of the weight tile,
+// 128 of the 256 weight rows (for SwiGLU: CTA 0 the gate rows, CTA 1 the up rows).  One thread of the
+// even CTA issues tcgen05.mma.cta_group::2 (M = 256, N = 256, K = 16): each SM's tensor core multiplies
+// its own A rows by the whole B tile, whose halves it reads from both CTAs' shared memory.  Per SM and
+// k-block that is 32 KB of TMA traffic instead of 48 KB, which lifts the shared-memory bound of the
+// one-SM kernel.  TMA loads of both CTAs signal the even CTA's mbarrier (cta_group::2 form, no multicast
+// load); stage release and accumulator hand-over reach both CTAs through multicast tcgen05.commit.
+// Persistent: cluster c works on pair-tiles c, c + #clusters, ... with the row tile fastest.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace d2c {
+namespace {
+
+constexpr int TM = 128, TK = 64;
+constexpr int TC_THREADS = 192;
+constexpr int A_BYTES = TM * TK * 2;             // 16 KB: this CTA's rows
+constexpr int BH_BYTES = 128 * TK * 2;           // 16 KB: this CTA's half of the weight tile
+constexpr int STAGE2 = A_BYTES + BH_BYTES;       // 32 KB per CTA and stage
+constexpr int ST2 = 6;
+constexpr int ACC_COLS = 256;
+constexpr long long kWaitCycles = 4000000000LL;
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;      // clears the CTA-rank bit of a shared::cluster address: the even CTA
+
+__device__ int g_tc_status[4];
+
+// ------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile("{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
+               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  return done;
+}
+// Bounded wait.  Returns false if it gave up (or another thread of the CTA already had).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = site;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                 "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                 "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                 "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte rows with the 128-byte
+// swizzle (what the TMA box load produces): 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);      // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+
+union Pack8 { uint4 u; __nv_bfloat162 h[4]; };
+
+
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
+// TMA load of one CTA of a pair; completion bytes go to the even CTA's barrier.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar & kPeerMask), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_even_cta(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
+}
+// bf16 x bf16 -> fp32, K-major operands, M = 256 across the pair, N = 256.
+constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+
+struct Tc2Params { GemmArgs g; int* status; };
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const __grid_constant__ CUtensorMap tmB2, const Tc2Params p) {
+  pdl_prologue();
+  constexpr int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : 256;  // output columns per pair-tile
+  const GemmArgs& g = p.g;
+  const int n = *g.n_rows;
+  if (n <= 0) return;
+  const int MT = (n + 2 * TM - 1) / (2 * TM), NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int total = MT * NT;
+  const int cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
+  if (cl >= total) return;                                   // same answer in both CTAs of a cluster
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KT = g.K / TK;
+  int* status = p.status ? p.status : g_tc_status;
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
+  __shared__ __align__(8) uint64_t bars[2 * ST2 + 4];        // full[ST2], empty[ST2], acc_full[2], acc_empty[2]
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (ST2 + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * ST2 + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * ST2 + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ST2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }   // 4 epilogue warps x 2 CTAs
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc2((uint32_t)__cvta_generic_to_shared(&tmem_slot), 2 * ACC_COLS);
+    tmem_relinquish2();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                        // both CTAs' barriers exist before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_slot;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = cl; tile < total && ok; tile += ncl) {
+        const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
+        const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : &tmB;
+        const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * 128;
+        for (int kt = 0; kt < KT; ++kt, ++it) {
+          const int s = it % ST2;
+          if (!mbar_wait(empty_bar(s), ((it / ST2) & 1) ^ 1, abortp, status, 31)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
+          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2);   // this CTA's two boxes and the peer's two
+          tma_load_2d_pair(sa, &tmA, kt * TK, m0, full_bar(s));
+          tma_load_2d_pair(sb, mb, kt * TK, brow, full_bar(s));
+        }
+      }
+      if (*abortp && leader) {
+        for (uint32_t j = it > (uint32_t)ST2 ? it - ST2 : 0; j < it; ++j) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full_bar(j % ST2), (j / ST2) & 1) && clock64() - t0 < kWaitCycles) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even CTA only)
+    if (lane == 0 && leader) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = cl; tile < total && ok; tile += ncl, ++tcount) {
+        const uint32_t buf = tcount & 1, use = tcount >> 1;
+        if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 34)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_acc + buf * ACC_COLS;
+        for (int kt = 0; kt < KT; ++kt, ++it) {
+          const int s = it % ST2;
+          if (!mbar_wait(full_bar(s), (it / ST2) & 1, abortp, status, 32)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < TK / 16; ++k)
+            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, kIdesc2, (kt | k) != 0);
+          umma2_commit_both(empty_bar(s));                    // both CTAs may refill this stage
+        }
+        if (ok) umma2_commit_both(acc_full(buf));             // both CTAs' epilogues may read their rows
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int quarter = warp & 3;
+    const int lrow = quarter * 32 + lane;
+    uint32_t tcount = 0;
+    for (int tile = cl; tile < total; tile += ncl, ++tcount) {
+      const uint32_t buf = tcount & 1, use = tcount >> 1;
+      const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
+      const int row = m0 + lrow;
+      const bool row_ok = row < n;
+      if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 33)) break;
+      tc_fence_after();
+      const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
+      auto load_chunk = [&](int col, uint32_t (&v)[32]) { tmem_ld32(tbase + col, v); tmem_ld_wait(); };
+      if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+        const bool vec = (g.ldc & 7) == 0;
+#pragma unroll 1
+        for (int c = 0; c < (OUT_COLS / 32); ++c) {
+          uint32_t v[32];
+          tmem_ld32(tbase + c * 32, v);
+          tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if (!row_ok || col0 >= g.N) continue;
+          bf16* dst = g.C + (size_t)row * g.ldc + col0;
+          if (vec && col0 + 32 <= g.N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              Pack8 o, old;
+              if (EPI == EPI_RESIDUAL) old.u = reinterpret_cast<const uint4*>(dst)[q];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
+                if (EPI == EPI_STORE) {
+                  if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
+                } else {
+                  const float2 of = __bfloat1622float2(old.h[e]);
+                  f0 += of.x; f1 += of.y;
+                }
+                o.h[e] = __floats2bfloat162_rn(f0, f1);
+              }
+              reinterpret_cast<uint4*>(dst)[q] = o.u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (col0 + j < g.N) {
+                float f = __uint_as_float(v[j]);
+                if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
+                else f += __bfloat162float(dst[j]);
+                dst[j] = __float2bfloat16_rn(f);
+              }
+            }
+          }
+        }
+      } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < (OUT_COLS / 32); ++c) {
+          uint32_t gv[32], uv[32];
+          tmem_ld32(tbase + c * 32, gv);
+          tmem_ld32(tbase + 128 + c * 32, uv);
+          tmem_ld_wait();
+          const int col0 = n0 + c * 32;
+          if (!row_ok || col0 >= g.N) continue;
+          bf16* dst = g.C + (size_t)row * g.ldc + col0;
+          if ((g.ldc & 7) == 0 && col0 + 32 <= g.N) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              Pack8 o;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float g0 = __uint_as_float(gv[q * 8 + 2 * e]), g1 = __uint_as_float(gv[q * 8 + 2 * e + 1]);
+                const float u0 = __uint_as_float(uv[q * 8 + 2 * e]), u1 = __uint_as_float(uv[q * 8 + 2 * e + 1]);
+                o.h[e] = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+              }
+              reinterpret_cast<uint4*>(dst)[q] = o.u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (col0 + j < g.N) {
+                const float gg = __uint_as_float(gv[j]), uu = __uint_as_float(uv[j]);
+                dst[j] = __float2bfloat16_rn(gg / (1.f + __expf(-gg)) * uu);
+              }
+            }
+          }
+        }
+      } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {         // statistics are kept per 128 columns
+          float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tbase + half * 128 + c * 32, v);
+            tmem_ld_wait();
+            const int col0 = n0 + half * 128 + c * 32;
+            if (col0 >= g.N) continue;
+            float cmx = -INFINITY; int carg = 0x7fffffff;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float f = __uint_as_float(v[j]);
+              if (col0 + j < g.N && f > cmx) { cmx = f; carg = col0 + j; }   // ascending columns: first maximum wins
+            }
+            const float nmx = fmaxf(mx, cmx);
+            float csum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < g.N) csum += __expf(__uint_as_float(v[j]) - nmx);
+            sum = sum * __expf(mx - nmx) + csum;                              // exp(-inf) = 0 on the first chunk
+            if (cmx > mx) arg = carg;
+            mx = nmx;
+            if (g.logits && row_ok) {
+              float* lp = g.logits + (size_t)row * g.N + col0;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < g.N) lp[j] = __uint_as_float(v[j]);
+            }
+          }
+          const int stile = nt * 2 + half;
+          if (row_ok && stile < g.n_tiles) {
+            const size_t o = (size_t)row * g.n_tiles + stile;
+            g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
+          }
+        }
+      }
+      // hand the accumulator back to the MMA thread in the even CTA
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_even_cta(acc_empty(buf));
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                        // nobody leaves while the peer may still signal it
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_acc, 2 * ACC_COLS);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D map over a row-major bf16 matrix [rows][cols] with leading dimension ld; box = box_rows x 64 columns,
+// 128-byte swizzle, out-of-range elements read as zero.
+int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) { set_global_error("cuTensorMapEncodeTiled is not available from this driver"); return D2C_ECUDA; }
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {TK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { set_global_error("cuTensorMapEncodeTiled failed with code %d", (int)r); return D2C_ECUDA; }
+  return D2C_OK;
+}
+
+
+int sm_count2() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+template <int EPI>
+int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
+  const int smem = ST2 * STAGE2 + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_set = true;
+  }
+  CUtensorMap tmA, tmB, tmB2;
+  int rc = make_map(&tmA, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
+  if (rc == D2C_OK) rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
+  if (rc == D2C_OK) rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
+  if (rc != D2C_OK) return rc;
+  Tc2Params p{g, status};
+  const int out_cols = EPI == EPI_SWIGLU ? 128 : 256;
+  const long long tiles = (long long)ceil_div(g.max_rows, 2 * TM) * ceil_div(g.N, out_cols);
+  const int pairs = (int)(tiles < sm_count2() / 2 ? tiles : sm_count2() / 2);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  D2C_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, tmB2, p));
+  count_launch(1);
+  return D2C_OK;
+}
+}  // namespace
+
+// Shapes the pair kernel takes; everything else goes to the one-SM kernel.
+bool gemm_tc2_supported(const GemmArgs& g) {
+  return g.max_rows >= 2 * TM && g.N >= 256 && g.K % TK == 0 && (g.lda & 7) == 0 && (g.N & 1) == 0 &&
+         (reinterpret_cast<uintptr_t>(g.A) & 15) == 0 && (reinterpret_cast<uintptr_t>(g.W) & 15) == 0;
+}
+
+int launch_gemm_tc2(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status) {
+  switch (epi) {
+    case EPI_STORE: return launch_one<EPI_STORE>(g, status, st);
+    case EPI_RESIDUAL: return launch_one<EPI_RESIDUAL>(g, status, st);
+    case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(g, status, st);
+    case EPI_LMSTATS: return launch_one<EPI_LMSTATS>(g, status, st);
+  }
+  return D2C_EINVAL;
+}
+
+}  // namespace d2c

@@ -62,8 +62,9 @@ int d2c_op_gemm(const void* A, const void* W, const void* bias, void* C, const i
   g.n_rows = n_rows; g.max_rows = max_rows; g.N = N; g.K = K;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (impl == 1) return launch_gemm_mma(g, EPI_STORE, st);
-  if (impl == 0) return launch_gemm_tc(g, EPI_STORE, st);
-  return bad(D2C_EINVAL, "d2c_op_gemm: impl must be 0 (tcgen05) or 1 (mma.sync)");
+  if (impl == 0) return gemm_tc2_supported(g) ? launch_gemm_tc2(g, EPI_STORE, st) : launch_gemm_tc(g, EPI_STORE, st);
+  if (impl == 2) return launch_gemm_tc(g, EPI_STORE, st);
+  return bad(D2C_EINVAL, "d2c_op_gemm: impl must be 0 (tcgen05), 1 (mma.sync) or 2 (one-SM tcgen05)");
 }
 
 int d2c_op_attention(const void* q, int32_t q_rows, int32_t ldq, const void* kcache, const void* vcache,
@@ -102,7 +103,7 @@ int d2c_op_lm_head(const void* x, const void* w_lm, const int32_t* n_rows, int32
   g.A = (const bf16*)x; g.lda = d; g.W = (const bf16*)w_lm; g.n_rows = n_rows; g.max_rows = max_rows; g.N = vocab; g.K = d;
   g.st_max = reinterpret_cast<float*>(sp); g.st_sum = reinterpret_cast<float*>(sp + piece);
   g.st_arg = reinterpret_cast<int32_t*>(sp + 2 * piece); g.n_tiles = nt; g.logits = logits;
-  int rc = launch_gemm_mma(g, EPI_LMSTATS, st);
+  int rc = launch_gemm_tc(g, EPI_LMSTATS, st);
   if (rc != D2C_OK) return rc;
   return launch_lm_reduce(g.st_max, g.st_sum, g.st_arg, nt, n_rows, max_rows, nullptr, nullptr, nullptr, 0, conf, pred, st);
 }

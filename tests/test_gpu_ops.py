@@ -16,7 +16,7 @@ def _bf16(shape, seed, std=1.0):
     return (torch.randn(*shape, generator=g) * std).to(torch.bfloat16)
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 2, 0])
 @pytest.mark.parametrize("rows,n,N,K", [(200, 200, 256, 128), (300, 131, 384, 256), (128, 128, 128, 64),
                                          (520, 517, 1000, 192), (64, 0, 256, 128), (260, 1, 128, 1024),
                                          (256, 100, 4096, 512), (1024, 130, 2048, 256), (512, 40, 8192, 128)])
