@@ -312,7 +312,7 @@ def oracle_setup(wl, w_cpu, mask, tokens):
     return ostep, wf, h0, st
 
 
-def cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L, max_rows=256):
+def cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L, max_rows=1024):
     """The oracle, as it stands, on the host cores: one partial step on a bounded sample of the rows."""
     if wl.shape.n_layers > 4:
         return {"value": None, "unit": UNIT, "kind": "oracle", "cores": os.cpu_count(),
@@ -355,7 +355,7 @@ def run_reference(args):
     st.conf[:] = rng.random(st.conf.shape).astype(np.float32)
     st.c[:] = (1.0 + 0.05 * rng.standard_normal(st.c.shape)).astype(np.float32)
     from oracle import selection as osel
-    rows_per_step = 96
+    rows_per_step = 256
     sample = []
     for b in range(B):
         S, _, _ = osel.select_rows(mask[b].numpy(), st.conf[b], st.c[b], wl.k, wl.p, wl.sigma)
