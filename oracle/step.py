@@ -68,11 +68,13 @@ def oracle_step(state: OracleState, w: Dict[str, object], shape, h0: np.ndarray,
                 k: int, p: float, sigma: float = 10.0,
                 forced: Optional[Sequence[Sequence[int]]] = None, stage2_candidates: int = 0,
                 sel_override: Optional[Sequence[np.ndarray]] = None,
-                rollout_literal: bool = False) -> StepResult:
+                rollout_literal: bool = False, rollout_layers: int = 0) -> StepResult:
     """One step.  h0: [B][L][d] input hidden states (embeddings of y_t), mask: [B][L] 1 = masked.
 
     `shape` needs n_q_heads, n_kv_heads, head_dim, rope_base, rms_eps.
     sel_override replaces step 1 with given index sets (teacher forcing in parity tests).
+    rollout_layers > 0 rolls the attention out over the first layers only (the paper's "Rollout-5"
+    variant, appendix table on rollout depth); 0 uses all layers (Eq. 8).
     The state is updated in place.
     """
     B, L, d = h0.shape
@@ -107,7 +109,8 @@ def oracle_step(state: OracleState, w: Dict[str, object], shape, h0: np.ndarray,
             lg = np.zeros((0, w["w_lm"].shape[0]))
         if S.size:
             cfun = rollout.literal if rollout_literal else rollout.chain
-            state.c[b] = cfun(abars, S, L).astype(np.float32)
+            depth = rollout_layers if 0 < rollout_layers < state.n_layers else state.n_layers
+            state.c[b] = cfun(abars[:depth], S, L).astype(np.float32)
         res.sel.append(S); res.m_star.append(m_star); res.u.append(u)
         res.hidden.append(x); res.abar.append(abars); res.lm_rows.append(lm_rows); res.logits.append(lg)
     return res

@@ -37,19 +37,20 @@ class Pair:
     """A CUDA context and an oracle state fed the same weights and inputs."""
 
     def __init__(self, wl: inputs.Workload, gain_jitter=0.05, std=0.02, stage2_candidates=0, rollout_layers=0,
-                 max_batch=None, max_seq=None):
+                 max_batch=None, max_seq=None, flags=0):
         self.wl, self.shape = wl, wl.shape
         self.w_cpu = inputs.make_weights(wl.shape, seed=wl.seed, gain_jitter=gain_jitter, std=std)
         self.w_dev = to_dev(self.w_cpu)
         self.wf = ostep.weights_to_f64(self.w_cpu)
         self.cfg = binding.make_config(wl.shape, max_batch or wl.batch, max_seq or wl.seq_len, sigma=wl.sigma,
-                                       stage2_candidates=stage2_candidates, rollout_layers=rollout_layers)
+                                       stage2_candidates=stage2_candidates, rollout_layers=rollout_layers, flags=flags)
         self.ctx = binding.Context(self.cfg, self.w_dev)
         self.ost = ostep.OracleState(wl.shape.n_layers, wl.batch, wl.seq_len, wl.shape.n_kv_heads, wl.shape.head_dim)
         self.mask = inputs.make_mask(wl)
         self.tokens = inputs.make_tokens(wl, self.mask)
         self.h0 = inputs.make_h0(self.w_cpu["embed"], self.tokens)
         self.stage2_candidates = stage2_candidates
+        self.rollout_layers = rollout_layers
 
     def gpu_step(self, k, p, forced=None, want_logits=False, mask=None, h0=None):
         wl = self.wl
@@ -93,4 +94,4 @@ class Pair:
         mask = self.mask if mask is None else mask
         h0 = self.h0 if h0 is None else h0
         return ostep.oracle_step(self.ost, self.wf, self.shape, h0.double().numpy(), mask.numpy(), k=0, p=0.0,
-                                 sigma=self.wl.sigma, sel_override=sel)
+                                 sigma=self.wl.sigma, sel_override=sel, rollout_layers=self.rollout_layers)

@@ -206,3 +206,32 @@ def test_decode_loop_commits_match_the_oracle_rule(rule):
         for b in range(B):
             assert row_rel_err(hid[ro[b]: ro[b + 1]].float().cpu().numpy(), res.hidden[b]) <= ROW_TOL
         fresh = [np.array([p for p in S[b] if got_mask[b, p]]) for b in range(B)]
+
+
+def test_truncated_rollout_depth():
+    """rollout_layers = 2 on a 3-layer model: the scores come from the first two layers' attention only."""
+    wl = WLS["gqa_bias_3layers"]
+    pair = Pair(wl, rollout_layers=2)
+    _prefill(pair)
+    g = pair.gpu_step(wl.k, wl.p)
+    res = pair.oracle_step(g["sel"])
+    _compare_state(pair, res, g["sel"])
+    full = Pair(wl)                                                   # same inputs, full depth: the scores must differ
+    _prefill(full)
+    assert not torch.allclose(full.ctx.view("c", wl.batch, wl.seq_len), pair.ctx.view("c", wl.batch, wl.seq_len), atol=1e-4)
+
+
+def test_kernel_variants_agree():
+    """The mma.sync GEMM / attention kernels and the one-SM tcgen05 GEMM give the same step within tolerance."""
+    wl = inputs.Workload("hd128_big", inputs.TOY_HD128, 2, 300, 150, 60, "random", 8, 0.6, seed=9)
+    ref = None
+    for flags in (0, 1 | 2, 4):                                       # default; portable GEMM + attention; one-SM GEMM
+        pair = Pair(wl, flags=flags)
+        pair.gpu_step(10 ** 6, 1.0)
+        g = pair.gpu_step(wl.k, wl.p)
+        if ref is None:
+            ref = g
+            continue
+        for b in range(wl.batch):
+            np.testing.assert_array_equal(g["sel"][b], ref["sel"][b])
+            assert row_rel_err(g["hidden"][b], ref["hidden"][b].astype(np.float64)) <= ROW_TOL
