@@ -140,23 +140,34 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_even_cta(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
 }
-// bf16 x bf16 -> fp32, K-major operands, M = 256 across the pair, N = 256.
-constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
 
 struct Tc2Params { GemmArgs g; int* status; };
 
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const __grid_constant__ CUtensorMap tmB2, const Tc2Params p) {
+                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmB64,
+                const __grid_constant__ CUtensorMap tmB32, const Tc2Params p) {
   pdl_prologue();
-  constexpr int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : 256;  // output columns per pair-tile
   const GemmArgs& g = p.g;
   const int n = *g.n_rows;
   if (n <= 0) return;
-  const int MT = (n + 2 * TM - 1) / (2 * TM), NT = (g.N + OUT_COLS - 1) / OUT_COLS;
-  const int total = MT * NT;
+  const int MT = (n + 2 * TM - 1) / (2 * TM);
   const int cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
+  // Accumulator width: 256 columns, halved (to 128, then 64) while the narrower tiling fills the last
+  // wave of clusters so much better that it outweighs the far less efficient narrow MMA (measured factor ~0.6).
+  int bn = ACC_COLS;
+  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+    while (bn > 64) {
+      const int t_wide = MT * ((g.N + bn - 1) / bn), t_narrow = MT * ((g.N + bn / 2 - 1) / (bn / 2));
+      const float e_wide = (float)t_wide / (float)(((t_wide + ncl - 1) / ncl) * ncl);
+      const float e_narrow = (float)t_narrow / (float)(((t_narrow + ncl - 1) / ncl) * ncl);
+      if (e_narrow * 0.6f > e_wide) bn >>= 1; else break;
+    }
+  }
+  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per pair-tile
+  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int total = MT * NT;
   if (cl >= total) return;                                   // same answer in both CTAs of a cluster
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
@@ -200,13 +211,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       bool ok = true;
       for (int tile = cl; tile < total && ok; tile += ncl) {
         const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
-        const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : &tmB;
-        const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * 128;
+        const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
+        const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
         for (int kt = 0; kt < KT; ++kt, ++it) {
           const int s = it % ST2;
           if (!mbar_wait(empty_bar(s), ((it / ST2) & 1) ^ 1, abortp, status, 31)) { ok = false; break; }
           const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
-          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2);   // this CTA's two boxes and the peer's two
+          if (leader) mbar_expect_tx(full_bar(s), 2 * (A_BYTES + (uint32_t)(bn / 2) * TK * 2));   // both CTAs' boxes
           tma_load_2d_pair(sa, &tmA, kt * TK, m0, full_bar(s));
           tma_load_2d_pair(sb, mb, kt * TK, brow, full_bar(s));
         }
@@ -224,6 +235,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (lane == 0 && leader) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((256u >> 4) << 24);
       for (int tile = cl; tile < total && ok; tile += ncl, ++tcount) {
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 34)) { ok = false; break; }
@@ -237,7 +249,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
 #pragma unroll
           for (int k = 0; k < TK / 16; ++k)
-            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, kIdesc2, (kt | k) != 0);
+            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
           umma2_commit_both(empty_bar(s));                    // both CTAs may refill this stage
         }
         if (ok) umma2_commit_both(acc_full(buf));             // both CTAs' epilogues may read their rows
@@ -436,13 +448,15 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_set = true;
   }
-  CUtensorMap tmA, tmB, tmB2;
+  CUtensorMap tmA, tmB, tmB2, tmB64, tmB32;
   int rc = make_map(&tmA, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
   if (rc == D2C_OK) rc = make_map(&tmB, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
   if (rc == D2C_OK) rc = make_map(&tmB2, EPI == EPI_SWIGLU ? g.W2 : g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 128);
+  if (rc == D2C_OK) rc = make_map(&tmB64, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 64);
+  if (rc == D2C_OK) rc = make_map(&tmB32, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 32);
   if (rc != D2C_OK) return rc;
   Tc2Params p{g, status};
-  const int out_cols = EPI == EPI_SWIGLU ? 128 : 256;
+  const int out_cols = (EPI == EPI_STORE || EPI == EPI_RESIDUAL) ? 64 : (EPI == EPI_SWIGLU ? 128 : 256);   // narrowest tile
   const long long tiles = (long long)ceil_div(g.max_rows, 2 * TM) * ceil_div(g.N, out_cols);
   const int pairs = (int)(tiles < sm_count2() / 2 ? tiles : sm_count2() / 2);
   cudaLaunchConfig_t cfg = {};
@@ -453,7 +467,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  D2C_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, tmB2, p));
+  D2C_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, tmB2, tmB64, tmB32, p));
   count_launch(1);
   return D2C_OK;
 }
