@@ -117,6 +117,16 @@ def algorithmic_work(shape, batch, L, n_b, n_m, rollout_layers):
     return flops, byts
 
 
+def aggregate_replicas(total_ms, e2e_s, rows, world, device):
+    """Whole-job numbers of `world` independent replicas: the slowest rank's times, the sum of the rows."""
+    if world <= 1:
+        return total_ms, e2e_s, rows
+    t = torch.tensor([total_ms, e2e_s, rows], dtype=torch.float64, device=device)
+    tmax = t.clone(); torch.distributed.all_reduce(tmax, op=torch.distributed.ReduceOp.MAX)
+    tsum = t.clone(); torch.distributed.all_reduce(tsum, op=torch.distributed.ReduceOp.SUM)
+    return float(tmax[0]), float(tmax[1]), float(tsum[2])
+
+
 def build_pair(wl, device):
     from paper_2509_23094_b200 import binding
     w_cpu = inputs.make_weights(wl.shape, seed=wl.seed, device=device if wl.shape.n_layers > 4 else "cpu")
@@ -210,14 +220,7 @@ def run_ours(args, rank, world, device):
     h2d = B * L * d * 2 + B * L
     d2h = (B + 1) * 4 + n * 4 + n * d * 2 + 2 * B * L * 4
 
-    # aggregate over ranks (independent replicas): max time, summed rows
-    t = torch.tensor([total_ms, e2e_s, float(n)], dtype=torch.float64, device=device)
-    if world > 1:
-        tmax = t.clone(); torch.distributed.all_reduce(tmax, op=torch.distributed.ReduceOp.MAX)
-        tsum = t.clone(); torch.distributed.all_reduce(tsum, op=torch.distributed.ReduceOp.SUM)
-        total_ms, e2e_s, n_all = float(tmax[0]), float(tmax[1]), float(tsum[2])
-    else:
-        n_all = float(n)
+    total_ms, e2e_s, n_all = aggregate_replicas(total_ms, e2e_s, float(n), world, device)
     ms_per_step = total_ms / args.steps
     value = n_all / (ms_per_step * 1e-3)
     e2e_value = n_all / (e2e_s / e2e_steps)
