@@ -93,7 +93,11 @@ struct GemmArgs {
   const int32_t* n_rows; int max_rows; int N; int K;
   // EPI_LMSTATS: per (row, 128-column tile) running max / sum of exp / arg-max, optional raw logits
   float* st_max; float* st_sum; int32_t* st_arg; float* logits; int n_tiles;
+  // split-K scratch of the one-SM tcgen05 kernel (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
+  // and as many zero-initialised arrival counters
+  float* sk_partials; int32_t* sk_counters; int sk_max_tiles;
 };
+static const int kSkMaxTiles = 160;
 int launch_gemm_mma(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st);
 
 // ---- attention (attention.cu) ----------------------------------------------------------------

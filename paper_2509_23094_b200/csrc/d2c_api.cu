@@ -44,6 +44,7 @@ struct Buffers {
   bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar;
   float *st_max, *st_sum; int32_t* st_arg;
   float *u0, *u1, *partial;
+  float* sk_partials; int32_t* sk_counters;
   float* abar_part; size_t abar_part_floats;
   bf16* h0_stage; uint8_t* mask_stage; int32_t *forced_stage, *forced_off_stage; float *okey_stage, *oc_stage;
   int32_t* committed_stage;
@@ -75,6 +76,7 @@ static size_t carve(const d2c_config& c, void* base, Buffers* out) {
   b.st_max = w.take<float>(R * nt); b.st_sum = w.take<float>(R * nt); b.st_arg = w.take<int32_t>(R * nt);
   b.u0 = w.take<float>(R); b.u1 = w.take<float>(R);
   b.partial = w.take<float>((size_t)kRolloutSplit * R + (R + 3) / 4);     // partial sums + selected-flag bytes
+  b.sk_partials = w.take<float>((size_t)kSkMaxTiles * 128 * 256); b.sk_counters = w.take<int32_t>(kSkMaxTiles);
   // scratch for the head-split of the abar kernel: only worth having when the (rows x keys) grid is small
   const size_t tiles_worst = (size_t)ceil_div((int)L, 128) * ceil_div((int)L, 128) * B;
   b.abar_part_floats = tiles_worst < 2 * 160 ? (size_t)8 * R * L : 0;
@@ -112,6 +114,9 @@ struct d2c_ctx {
   cudaStream_t stream;
   Buffers buf;
   int phi_len;
+  // Selected-row count of an earlier step, copied to pinned host memory at the end of every step and read
+  // without synchronising: only a hint for choosing between GEMM kernels (both are correct for any count).
+  int32_t* n_hint = nullptr;
   char err[512];
   // optional per-phase timing: one event at every phase boundary, resolved by d2c_profile_read
   bool prof = false;
@@ -157,9 +162,12 @@ static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->stream);
   // The LM head runs on few rows and is bound by the weight stream: the one-SM kernel sizes its A boxes to the
   // live rows, a pair would load a second, empty row tile.
-  if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && gemm_tc2_supported(g))
+  const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;   // weight-streaming regime
+  if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && !few_rows && gemm_tc2_supported(g))
     return launch_gemm_tc2(g, epi, ctx->stream, ctx->buf.status);
-  return launch_gemm_tc(g, epi, ctx->stream, ctx->buf.status);
+  GemmArgs gs = g;
+  gs.sk_partials = ctx->buf.sk_partials; gs.sk_counters = ctx->buf.sk_counters; gs.sk_max_tiles = kSkMaxTiles;
+  return launch_gemm_tc(gs, epi, ctx->stream, ctx->buf.status);
 }
 #define D2C_TRY(ctx, expr) do { int rc__ = (expr); if (rc__ != D2C_OK) return pass((ctx), rc__); } while (0)
 
@@ -199,6 +207,8 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
   }
   ctx->g_final = (const bf16*)w->g_final; ctx->w_lm = (const bf16*)w->w_lm;
   carve(*cfg, workspace, &ctx->buf);
+  if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->n_hint), sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess) *ctx->n_hint = 1 << 30;
+  else { ctx->n_hint = nullptr; (void)cudaGetLastError(); }
   cudaError_t e = cudaMemsetAsync(workspace, 0, need, ctx->stream);
   if (e == cudaSuccess) {
     std::vector<uint32_t> tab(cfg->max_seq);
@@ -218,6 +228,7 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
 int d2c_destroy(d2c_ctx* ctx) {
   if (!ctx) return D2C_EINVAL;
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+  if (ctx->n_hint) cudaFreeHost(ctx->n_hint);
   delete ctx;
   return D2C_OK;
 }
@@ -355,6 +366,10 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   }
   if (out && out->row_off) {
     cudaError_t e = cudaMemcpyAsync(out->row_off, b.row_off, (size_t)(B + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
+  }
+  if (ctx->n_hint) {
+    cudaError_t e = cudaMemcpyAsync(ctx->n_hint, b.row_off + B, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
   }
   D2C_TRY(ctx, mark(ctx, -1));

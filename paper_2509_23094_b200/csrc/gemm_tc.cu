@@ -113,7 +113,8 @@ struct TcParams {
   int* status;
 };
 
-constexpr int ST = 4;                            // shared-memory stages: 4 x (16 KB of A + 32 KB of B)
+constexpr int ST = 4;                            // stages at full tile width: 4 x (16 KB of A + 32 KB of B)
+constexpr int ST_MAX = 12;                       // narrow tiles use smaller stages and more of them
 constexpr int ACC_COLS = 256;                    // TMEM columns of one accumulator; two are allocated
 constexpr int B_BYTES = ACC_COLS * TK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -145,24 +146,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
   const int total = MT * NT;
-  if ((int)blockIdx.x >= total) return;                      // uniform: nothing allocated yet
+  const int KT = g.K / TK, G = gridDim.x;
+  // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
+  // idle SM is lost bandwidth): each tile's K range is cut into S equal parts handled by different CTAs.
+  // Parts park their fp32 accumulators in scratch; the part that arrives last adds them in part order
+  // (no waiting, deterministic) and runs the epilogue.
+  int S = 1;
+  if (g.sk_partials != nullptr && g.sk_counters != nullptr && total < G && total <= g.sk_max_tiles)
+    S = max(1, min(min(G / total, KT / 8), 4));
+  const int items = total * S;
+  if ((int)blockIdx.x >= items) return;                      // uniform: nothing allocated yet
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int KT = g.K / TK;
   int* status = p.status ? p.status : g_tc_status;
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
-  __shared__ __align__(8) uint64_t bars[2 * ST + 4];         // full[ST], empty[ST], acc_full[2], acc_empty[2]
+  __shared__ __align__(8) uint64_t bars[2 * ST_MAX + 4];     // full[], empty[], acc_full[2], acc_empty[2]
   __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag, sk_last;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (ST + s); };
-  auto acc_full = [&](int b) { return bar0 + 8u * (2 * ST + b); };
-  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * ST + 2 + b); };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (ST_MAX + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * ST_MAX + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * ST_MAX + 2 + b); };
+  // Stage size follows the tile this launch uses (A box of 128 rows or less, bn weight rows); the freed
+  // shared memory becomes more stages, i.e. more bytes in flight per SM when the launch streams weights.
+  const int a_rows_max = n >= 128 ? 128 : (n > 64 ? 128 : (n > 32 ? 64 : 32));
+  const int stage_bytes = ((a_rows_max + ((EPI == EPI_SWIGLU) ? ACC_COLS : bn)) * TK * 2 + 1023) & ~1023;
+  // the MMA always reads 128 rows of A: keep that read inside the allocation when the A box is smaller
+  const int nst = min(ST_MAX, (ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2) / stage_bytes);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < ST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < nst; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -183,15 +198,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     if (lane == 0) {
       uint32_t it = 0;                                        // k-blocks issued so far (ring position)
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+      for (int item = blockIdx.x; item < items && ok; item += G) {
+        const int tile = item % total, part = item / total;
+        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const int m0 = (tile % MT) * TM, n0 = (tile / MT) * OUT_COLS;
         const int rows = n - m0;                              // live rows of this tile: load no more than needed
         const CUtensorMap* ma = rows <= 32 ? &tmA32 : (rows <= 64 ? &tmA64 : &tmA128);
         const uint32_t a_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2;
-        for (int kt = 0; kt < KT; ++kt, ++it) {
-          const int s = it % ST;
-          if (!mbar_wait(empty_bar(s), ((it / ST) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
-          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+        for (int kt = k0; kt < k1; ++kt, ++it) {
+          const int s = it % nst;
+          if (!mbar_wait(empty_bar(s), ((it / nst) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * stage_bytes, sb = sa + a_rows_max * TK * 2;
           mbar_expect_tx(full_bar(s), a_bytes + (uint32_t)bn * TK * 2);
           tma_load_2d(sa, ma, kt * TK, m0, full_bar(s));
           if (bn == 64) {
@@ -205,9 +222,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       }
       if (*abortp) {
         // give the copies already in flight a bounded chance to land before the CTA goes away
-        for (uint32_t j = it > (uint32_t)ST ? it - ST : 0; j < it; ++j) {
+        for (uint32_t j = it > (uint32_t)nst ? it - nst : 0; j < it; ++j) {
           const long long t0 = clock64();
-          while (!mbar_try_wait(full_bar(j % ST), (j / ST) & 1) && clock64() - t0 < kWaitCycles) {}
+          while (!mbar_try_wait(full_bar(j % nst), (j / nst) & 1) && clock64() - t0 < kWaitCycles) {}
         }
       }
     }
@@ -218,20 +235,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       const uint32_t idesc = instr_desc(bn);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++tcount) {
+      for (int item = blockIdx.x; item < items && ok; item += G, ++tcount) {
+        const int part = item / total;
+        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 4)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
-        for (int kt = 0; kt < KT; ++kt, ++it) {
-          const int s = it % ST;
-          if (!mbar_wait(full_bar(s), (it / ST) & 1, abortp, status, 2)) { ok = false; break; }
+        for (int kt = k0; kt < k1; ++kt, ++it) {
+          const int s = it % nst;
+          if (!mbar_wait(full_bar(s), (it / nst) & 1, abortp, status, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint32_t sa = smem_base + s * stage_bytes, sb = sa + a_rows_max * TK * 2;
           const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
 #pragma unroll
           for (int k = 0; k < TK / 16; ++k)                   // +32 bytes per K=16 slice inside the swizzle atom
-            umma_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+            umma_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, ((kt - k0) | k) != 0);
           umma_commit(empty_bar(s));                          // stage reusable once these MMAs have read it
         }
         if (ok) umma_commit(acc_full(buf));                   // accumulator complete
@@ -243,7 +262,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     const int quarter = warp & 3;                             // TMEM lanes this warp may touch
     const int lrow = quarter * 32 + lane;
     uint32_t tcount = 0;
-    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++tcount) {
+    for (int item = blockIdx.x; item < items; item += G, ++tcount) {
+      const int tile = item % total, part = item / total;
       const uint32_t buf = tcount & 1, use = tcount >> 1;
       const int m0 = (tile % MT) * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int n_chunks = OUT_COLS / 32;
@@ -252,13 +272,67 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 3)) break;
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
+      bool reduce = false;
+      if (S > 1) {
+        const int acc_cols = (EPI == EPI_SWIGLU) ? ACC_COLS : bn;
+        float4* mine = reinterpret_cast<float4*>(g.sk_partials + (size_t)(tile * S + part) * (TM * ACC_COLS));
+#pragma unroll 1
+        for (int c = 0; c < acc_cols / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tbase + c * 32, v);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              mine[(size_t)(c * 8 + q) * TM + lrow] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                                  __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          }
+        }
+        tc_fence_before();
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf));
+          const int old = atomicAdd(&g.sk_counters[tile], 1);
+          const int last = (old == S - 1) ? 1 : 0;
+          if (last) g.sk_counters[tile] = 0;                 // every part has arrived: ready for the next launch
+          sk_last = last;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        reduce = sk_last != 0;
+        asm volatile("bar.sync 1, 128;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
+        if (!reduce) continue;
+        __threadfence();
+      }
+      auto load_chunk = [&](int col, uint32_t (&v)[32]) {     // 32 accumulator columns of this thread's row
+        if (!reduce) {
+          tmem_ld32(tbase + col, v);
+          tmem_ld_wait();
+        } else {
+          float4 t[4][8];
+          const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + (size_t)(tile * S) * (TM * ACC_COLS)) +
+                             (size_t)(col >> 2) * TM + lrow;
+#pragma unroll
+          for (int c2 = 0; c2 < 4; ++c2)
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              t[c2][q] = (c2 < S && row_ok) ? __ldcg(sp + (size_t)c2 * (TM * ACC_COLS / 4) + (size_t)q * TM) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 acc = t[0][q];
+#pragma unroll
+            for (int c2 = 1; c2 < 4; ++c2) { acc.x += t[c2][q].x; acc.y += t[c2][q].y; acc.z += t[c2][q].z; acc.w += t[c2][q].w; }
+            v[4 * q] = __float_as_uint(acc.x); v[4 * q + 1] = __float_as_uint(acc.y);
+            v[4 * q + 2] = __float_as_uint(acc.z); v[4 * q + 3] = __float_as_uint(acc.w);
+          }
+        }
+      };
       if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < n_chunks; ++c) {
           uint32_t v[32];
-          tmem_ld32(tbase + c * 32, v);
-          tmem_ld_wait();
+          load_chunk(c * 32, v);
           const int col0 = n0 + c * 32;
           if (!row_ok || col0 >= g.N) continue;
           bf16* dst = g.C + (size_t)row * g.ldc + col0;
@@ -296,9 +370,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
 #pragma unroll 1
         for (int c = 0; c < n_chunks; ++c) {
           uint32_t gv[32], uv[32];
-          tmem_ld32(tbase + c * 32, gv);
-          tmem_ld32(tbase + 128 + c * 32, uv);
-          tmem_ld_wait();
+          load_chunk(c * 32, gv);
+          load_chunk(128 + c * 32, uv);
           const int col0 = n0 + c * 32;
           if (!row_ok || col0 >= g.N) continue;
           bf16* dst = g.C + (size_t)row * g.ldc + col0;
@@ -331,8 +404,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             uint32_t v[32];
-            tmem_ld32(tbase + half * 128 + c * 32, v);
-            tmem_ld_wait();
+            load_chunk(half * 128 + c * 32, v);
             const int col0 = n0 + half * 128 + c * 32;
             if (col0 >= g.N) continue;
             float cmx = -INFINITY; int carg = 0x7fffffff;
@@ -363,10 +435,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
           }
         }
       }
-      // hand the accumulator back to the MMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty(buf));
+      // hand the accumulator back to the MMA warp (a split-K part has done so already)
+      if (!reduce) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty(buf));
+      }
     }
   }
   // ------------------------------------------------------------------ teardown
