@@ -109,6 +109,9 @@ typedef struct {
   float   p;                       /* top-p threshold; <= 0 selects nothing, >= 1 every candidate         */
   const float* override_key;       /* optional [batch][seq_len]: use as stage-1 keys instead of D(i)*s^i  */
   const float* override_c;         /* optional [batch][seq_len]: use as stage-2 scores instead of state c */
+  int32_t block_lo, block_hi;      /* semi-autoregressive decoding (blocks decoded left to right, Section 5.1):
+                                      stage 1 only considers masked positions in [block_lo, block_hi);
+                                      block_hi <= block_lo means the whole sequence                        */
 } d2c_step_args;
 
 typedef struct {

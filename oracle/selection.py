@@ -91,13 +91,20 @@ def _clean_score(x: np.ndarray) -> np.ndarray:
 
 
 def stage1_select(mask: np.ndarray, conf: np.ndarray, k: int, sigma: float,
-                  key: Optional[np.ndarray] = None) -> np.ndarray:
-    """Eq. 4: indices of the k largest keys over the masked set (all of it if it has <= k members)."""
+                  key: Optional[np.ndarray] = None, block: Optional[Tuple[int, int]] = None) -> np.ndarray:
+    """Eq. 4: indices of the k largest keys over the masked set (all of it if it has <= k members).
+
+    block = (lo, hi) confines the masked set to positions lo <= i < hi: the reading taken here of
+    "semi-autoregressive decoding with d2Cache" (blocks decoded left to right, Section 5.1), which
+    the paper does not spell out.  The density of Eq. 3 still sees the whole sequence.
+    """
     mask = np.asarray(mask).astype(bool)
     if key is None:
         key = stage1_keys(mask, conf, sigma)
     key = _clean_score(key)
     members = [int(i) for i in np.flatnonzero(mask)]
+    if block is not None and block[1] > block[0]:
+        members = [i for i in members if block[0] <= i < block[1]]
     members.sort(key=lambda i: (-float(key[i]), i))
     return np.array(sorted(members[: max(0, int(k))]), dtype=np.int64)
 
@@ -125,7 +132,8 @@ def stage2_select(c: np.ndarray, candidates: np.ndarray, p: float) -> np.ndarray
 
 def select_rows(mask: np.ndarray, conf: np.ndarray, c: np.ndarray, k: int, p: float, sigma: float,
                 forced: Iterable[int] = (), stage2_candidates: int = 0,
-                key: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+                key: Optional[np.ndarray] = None, block: Optional[Tuple[int, int]] = None
+                ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """Both stages and their union (the index set of Eq. 5), for one sequence.
 
     stage2_candidates = 0: candidates are the known (prompt / decoded) positions;
@@ -133,7 +141,7 @@ def select_rows(mask: np.ndarray, conf: np.ndarray, c: np.ndarray, k: int, p: fl
     Returns (S ascending, M* ascending, U ascending).
     """
     mask = np.asarray(mask).astype(bool)
-    m_star = stage1_select(mask, conf, k, sigma, key=key)
+    m_star = stage1_select(mask, conf, k, sigma, key=key, block=block)
     if stage2_candidates == 0:
         cand = ~mask
     else:

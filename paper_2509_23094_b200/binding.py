@@ -45,7 +45,7 @@ class Weights(C.Structure):
 class StepArgs(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seq_len", C.c_int32), ("h0", C.c_void_p), ("mask", C.c_void_p),
                 ("forced", C.c_void_p), ("forced_off", C.c_void_p), ("k", C.c_int32), ("p", C.c_float),
-                ("override_key", C.c_void_p), ("override_c", C.c_void_p)]
+                ("override_key", C.c_void_p), ("override_c", C.c_void_p), ("block_lo", C.c_int32), ("block_hi", C.c_int32)]
 
 
 class StepOut(C.Structure):
@@ -218,10 +218,12 @@ class Context:
              forced_off: Optional[torch.Tensor] = None, override_key: Optional[torch.Tensor] = None,
              override_c: Optional[torch.Tensor] = None, hidden_out: Optional[torch.Tensor] = None,
              sel_idx: Optional[torch.Tensor] = None, row_off: Optional[torch.Tensor] = None,
-             logits: Optional[torch.Tensor] = None, layer_in: Optional[torch.Tensor] = None) -> None:
+             logits: Optional[torch.Tensor] = None, layer_in: Optional[torch.Tensor] = None,
+             block: Optional[Sequence[int]] = None) -> None:
         B, L = mask.shape
+        lo, hi = (int(block[0]), int(block[1])) if block is not None else (0, 0)
         a = StepArgs(B, L, _ptr(h0), _ptr(mask), _ptr(forced), _ptr(forced_off), int(k), float(p),
-                     _ptr(override_key), _ptr(override_c))
+                     _ptr(override_key), _ptr(override_c), lo, hi)
         o = StepOut(_ptr(sel_idx), _ptr(row_off), _ptr(hidden_out), _ptr(logits), _ptr(layer_in))
         _check(load().d2c_step(self.handle, C.byref(a), C.byref(o)), self.handle)
 
@@ -232,7 +234,7 @@ class Context:
             assert t is None or not t.is_cuda, "step_host takes host tensors"
         B, L = mask.shape
         a = StepArgs(B, L, _ptr(h0), _ptr(mask), _ptr(forced), _ptr(forced_off), int(k), float(p),
-                     _ptr(override_key), _ptr(override_c))
+                     _ptr(override_key), _ptr(override_c), 0, 0)
         o = HostOut(_ptr(sel_idx), _ptr(row_off), _ptr(hidden_out), _ptr(conf), _ptr(pred))
         _check(load().d2c_step_host(self.handle, C.byref(a), C.byref(o)), self.handle)
 

@@ -63,6 +63,7 @@ struct SelectArgs {
   const uint8_t* mask; const float* conf; const float* c; const float* override_key;
   const int32_t* forced; const int32_t* forced_off;
   int batch, seq_len, k; float p; int stage2_candidates;
+  int block_lo, block_hi;                        // stage 1 only looks at masked positions in [block_lo, block_hi); empty = all
   const uint32_t* phi_q30; int phi_len;          // phi table in 2^-30 fixed point, entries [0, phi_len)
   float* key; int32_t* sel_idx; int32_t* row_seq; int32_t* row_off; int32_t* lm_rows; int32_t* lm_off;
   int32_t* slot_of_pos;

@@ -284,7 +284,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   SelectArgs s{};
   s.mask = a->mask; s.conf = b.conf; s.c = a->override_c ? a->override_c : b.c; s.override_key = a->override_key;
   s.forced = a->forced; s.forced_off = a->forced_off; s.batch = B; s.seq_len = L; s.k = a->k; s.p = a->p;
-  s.stage2_candidates = c.stage2_candidates; s.phi_q30 = b.phi; s.phi_len = ctx->phi_len < L ? ctx->phi_len : L;
+  s.stage2_candidates = c.stage2_candidates; s.block_lo = a->block_lo; s.block_hi = a->block_hi; s.phi_q30 = b.phi; s.phi_len = ctx->phi_len < L ? ctx->phi_len : L;
   s.key = b.key; s.sel_idx = b.sel_idx; s.row_seq = b.row_seq; s.row_off = b.row_off; s.lm_rows = b.lm_rows;
   s.lm_off = b.lm_off; s.slot_of_pos = b.slot_of_pos; s.rank_s = b.rank_s; s.rank_lm = b.rank_lm; s.n_b = b.n_b; s.nm_b = b.nm_b;
   D2C_TRY(ctx, mark(ctx, PH_SELECT));

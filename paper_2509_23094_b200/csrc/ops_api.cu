@@ -47,7 +47,7 @@ int d2c_op_select(const uint8_t* mask, const float* conf, const float* c, const 
   D2C_CUDA_OK(cudaMemcpyAsync(phi, tab.data(), tab.size() * 4, cudaMemcpyHostToDevice, st));
   D2C_CUDA_OK(cudaStreamSynchronize(st));       // pageable host table: the copy must finish before it dies
   a.mask = mask; a.conf = conf; a.c = c; a.override_key = override_key; a.forced = forced; a.forced_off = forced_off;
-  a.batch = batch; a.seq_len = seq_len; a.k = k; a.p = p; a.stage2_candidates = stage2_candidates;
+  a.batch = batch; a.seq_len = seq_len; a.k = k; a.p = p; a.stage2_candidates = stage2_candidates; a.block_lo = 0; a.block_hi = 0;
   a.phi_q30 = phi; a.phi_len = phi_len;
   a.key = key; a.sel_idx = sel_idx; a.row_off = row_off; a.lm_rows = lm_rows; a.lm_off = lm_off; a.slot_of_pos = slot_of_pos;
   return launch_select(a, st);

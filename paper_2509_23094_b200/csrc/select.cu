@@ -82,6 +82,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
   const float* cs = a.c + (size_t)b * L;
   const float* okey = a.override_key ? a.override_key + (size_t)b * L : nullptr;
 
+  // stage 1 may be confined to one block of positions (semi-autoregressive decoding); whole sequence otherwise
+  const int blk_lo = a.block_hi > a.block_lo ? a.block_lo : 0, blk_hi = a.block_hi > a.block_lo ? a.block_hi : L;
   for (int i = tid; i < L; i += kSelThreads) { smask[i] = mask[i] ? 1 : 0; flags[i] = 0; }
   if (tid == 0) { s_cnt = 0; }
   __syncthreads();
@@ -93,7 +95,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
       uint64_t comp = 0;
       if (i < L) {
         float key = 0.f;
-        if (smask[i]) {
+        if (smask[i] && i >= blk_lo && i < blk_hi) {
           if (okey) {
             key = clean_score(okey[i]);
           } else {
@@ -109,9 +111,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
             key = clean_score(__fmul_rn(D, conf[i]));
           }
           comp = (1ull << 63) | ((uint64_t)__float_as_uint(key) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
-        } else {
+        } else if (!smask[i]) {
           comp = ((uint64_t)__float_as_uint(clean_score(cs[i])) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
-        }
+        }                                                           // masked outside the block: in neither stage
         a.key[(size_t)b * L + i] = key;
       }
       sbuf[i] = comp;
@@ -172,7 +174,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
     uint64_t comp = 0;
     if (i < L) {
       float key = 0.f;
-      if (smask[i]) {
+      if (smask[i] && i >= blk_lo && i < blk_hi) {
         if (okey) {
           key = clean_score(okey[i]);
         } else {

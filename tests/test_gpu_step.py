@@ -235,3 +235,26 @@ def test_kernel_variants_agree():
         for b in range(wl.batch):
             np.testing.assert_array_equal(g["sel"][b], ref["sel"][b])
             assert row_rel_err(g["hidden"][b], ref["hidden"][b].astype(np.float64)) <= ROW_TOL
+
+
+def test_semi_autoregressive_block_restricts_stage1():
+    from oracle import selection as osel
+    wl = inputs.Workload("semiar", inputs.TOY_HD128, 2, 192, 64, 128, "all", 6, 0.4, seed=5)
+    pair = Pair(wl)
+    _prefill(pair)
+    B, L = wl.batch, wl.seq_len
+    conf = pair.ctx.view("conf", B, L).cpu().numpy().copy(); c = pair.ctx.view("c", B, L).cpu().numpy().copy()
+    hid = torch.zeros(B * L, wl.shape.d_model, dtype=torch.bfloat16, device="cuda")
+    pair.ctx.step(pair.h0.cuda(), pair.mask.cuda(), wl.k, wl.p, hidden_out=hid, block=(96, 128))
+    pair.ctx.sync_status()
+    ro = pair.ctx.view("row_off", B, L).cpu().numpy(); sel = pair.ctx.view("sel_idx").cpu().numpy()
+    S = []
+    for b in range(B):
+        want, m_star, _ = osel.select_rows(pair.mask[b].numpy(), conf[b], c[b], wl.k, wl.p, wl.sigma, block=(96, 128))
+        got = sel[ro[b]: ro[b + 1]]
+        np.testing.assert_array_equal(got, want)
+        assert len(m_star) == wl.k and all(96 <= i < 128 for i in m_star)
+        S.append(got.astype(np.int64))
+    res = pair.oracle_step(S)
+    for b in range(B):
+        assert row_rel_err(hid[ro[b]: ro[b + 1]].float().cpu().numpy(), res.hidden[b]) <= ROW_TOL

@@ -204,3 +204,16 @@ def test_select_rows_union_and_candidate_modes():
     assert S.tolist() == list(range(L))
     S, _, _ = sel.select_rows(mask, conf, c, 0, 0.0, 10.0)
     assert S.size == 0
+
+
+def test_stage1_block_restriction():
+    mask = np.zeros(128, dtype=np.uint8); mask[64:] = 1
+    conf = np.linspace(0.1, 0.9, 128).astype(np.float32)          # later positions are more confident
+    whole = sel.stage1_select(mask, conf, 4, 10.0)
+    blocked = sel.stage1_select(mask, conf, 4, 10.0, block=(64, 96))
+    assert all(64 <= i < 96 for i in blocked) and len(blocked) == 4
+    assert blocked.tolist() == _rank_topk(np.where(np.arange(128) < 96, mask, 0), sel.stage1_keys(mask, conf, 10.0), 4).tolist()
+    assert sel.stage1_select(mask, conf, 4, 10.0, block=(5, 5)).tolist() == whole.tolist()     # empty block = no restriction
+    assert sel.stage1_select(mask, conf, 100, 10.0, block=(64, 70)).tolist() == list(range(64, 70))
+    S, m_star, u = sel.select_rows(mask, conf, np.ones(128, np.float32), 4, 0.1, 10.0, block=(64, 96))
+    assert m_star.tolist() == blocked.tolist() and all(j < 64 for j in u)
