@@ -164,7 +164,11 @@ static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   // live rows, a pair would load a second, empty row tile.
   const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;   // weight-streaming regime
   if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && !few_rows && gemm_tc2_supported(g))
-    return launch_gemm_tc2(g, epi, ctx->stream, ctx->buf.status);
+  {
+    GemmArgs g2 = g;
+    g2.sk_partials = ctx->buf.sk_partials; g2.sk_counters = ctx->buf.sk_counters; g2.sk_max_tiles = kSkMaxTiles;
+    return launch_gemm_tc2(g2, epi, ctx->stream, ctx->buf.status);
+  }
   GemmArgs gs = g;
   gs.sk_partials = ctx->buf.sk_partials; gs.sk_counters = ctx->buf.sk_counters; gs.sk_max_tiles = kSkMaxTiles;
   return launch_gemm_tc(gs, epi, ctx->stream, ctx->buf.status);

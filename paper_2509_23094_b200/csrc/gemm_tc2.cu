@@ -157,7 +157,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   // Accumulator width: 256 columns, halved (to 128, then 64) while the narrower tiling fills the last
   // wave of clusters so much better that it outweighs the far less efficient narrow MMA (measured factor ~0.6).
   int bn = ACC_COLS;
-  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+  const int KT = g.K / TK;
+  const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
+  const int t256 = MT * ((g.N + (EPI == EPI_SWIGLU ? 128 : 256) - 1) / (EPI == EPI_SWIGLU ? 128 : 256));
+  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;   // split-K beats narrow tiles
+  if ((EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split) {
     while (bn > 64) {
       const int t_wide = MT * ((g.N + bn - 1) / bn), t_narrow = MT * ((g.N + bn / 2 - 1) / (bn / 2));
       const float e_wide = (float)t_wide / (float)(((t_wide + ncl - 1) / ncl) * ncl);
@@ -168,18 +172,24 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per pair-tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
   const int total = MT * NT;
-  if (cl >= total) return;                                   // same answer in both CTAs of a cluster
+  // Split-K when there are fewer pair-tiles than clusters: K is cut into S equal parts, one (tile, part)
+  // item per cluster; every CTA parks its 128 rows of fp32 partial sums in scratch and, per (tile, CTA
+  // rank), the part that arrives last adds all parts in part order (no waiting, deterministic).
+  int S = 1;
+  if (sk_ok && total < ncl && 2 * total <= g.sk_max_tiles)
+    S = max(1, min(min(ncl / total, KT / 8), 4));
+  const int items = total * S;
+  if (cl >= items) return;                                   // same answer in both CTAs of a cluster
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int KT = g.K / TK;
   int* status = p.status ? p.status : g_tc_status;
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
   __shared__ __align__(8) uint64_t bars[2 * ST2 + 4];        // full[ST2], empty[ST2], acc_full[2], acc_empty[2]
   __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag, sk_last;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (ST2 + s); };
@@ -209,11 +219,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = cl; tile < total && ok; tile += ncl) {
+      for (int item = cl; item < items && ok; item += ncl) {
+        const int tile = item % total, part = item / total;
+        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
         const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
         const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
-        for (int kt = 0; kt < KT; ++kt, ++it) {
+        for (int kt = k0; kt < k1; ++kt, ++it) {
           const int s = it % ST2;
           if (!mbar_wait(empty_bar(s), ((it / ST2) & 1) ^ 1, abortp, status, 31)) { ok = false; break; }
           const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
@@ -236,12 +248,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((256u >> 4) << 24);
-      for (int tile = cl; tile < total && ok; tile += ncl, ++tcount) {
+      for (int item = cl; item < items && ok; item += ncl, ++tcount) {
+        const int part = item / total;
+        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 34)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
-        for (int kt = 0; kt < KT; ++kt, ++it) {
+        for (int kt = k0; kt < k1; ++kt, ++it) {
           const int s = it % ST2;
           if (!mbar_wait(full_bar(s), (it / ST2) & 1, abortp, status, 32)) { ok = false; break; }
           tc_fence_after();
@@ -249,7 +263,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
 #pragma unroll
           for (int k = 0; k < TK / 16; ++k)
-            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) != 0);
+            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, ((kt - k0) | k) != 0);
           umma2_commit_both(empty_bar(s));                    // both CTAs may refill this stage
         }
         if (ok) umma2_commit_both(acc_full(buf));             // both CTAs' epilogues may read their rows
@@ -261,7 +275,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;
     uint32_t tcount = 0;
-    for (int tile = cl; tile < total; tile += ncl, ++tcount) {
+    for (int item = cl; item < items; item += ncl, ++tcount) {
+      const int tile = item % total, part = item / total;
       const uint32_t buf = tcount & 1, use = tcount >> 1;
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
@@ -269,14 +284,68 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 33)) break;
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
-      auto load_chunk = [&](int col, uint32_t (&v)[32]) { tmem_ld32(tbase + col, v); tmem_ld_wait(); };
+      bool reduce = false;
+      const size_t slot_floats = (size_t)TM * ACC_COLS;
+      if (S > 1) {
+        const int acc_cols = (EPI == EPI_SWIGLU) ? ACC_COLS : bn;
+        float4* mine = reinterpret_cast<float4*>(g.sk_partials + ((size_t)(tile * S + part) * 2 + rank) * slot_floats);
+#pragma unroll 1
+        for (int c = 0; c < acc_cols / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tbase + c * 32, v);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              mine[(size_t)(c * 8 + q) * TM + lrow] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                                  __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          }
+        }
+        tc_fence_before();
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          for (int w4 = 0; w4 < 4; ++w4) mbar_arrive_even_cta(acc_empty(buf));
+          const int old = atomicAdd(&g.sk_counters[tile * 2 + rank], 1);
+          const int last = (old == S - 1) ? 1 : 0;
+          if (last) g.sk_counters[tile * 2 + rank] = 0;      // every part has arrived: ready for the next launch
+          sk_last = last;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        reduce = sk_last != 0;
+        asm volatile("bar.sync 1, 128;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
+        if (!reduce) continue;
+        __threadfence();
+      }
+      auto load_chunk = [&](int col, uint32_t (&v)[32]) {     // 32 accumulator columns of this thread's row
+        if (!reduce) {
+          tmem_ld32(tbase + col, v);
+          tmem_ld_wait();
+        } else {
+          float4 t[4][8];
+          const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + ((size_t)(tile * S) * 2 + rank) * slot_floats) +
+                             (size_t)(col >> 2) * TM + lrow;
+#pragma unroll
+          for (int c2 = 0; c2 < 4; ++c2)
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              t[c2][q] = (c2 < S && row_ok) ? __ldcg(sp + (size_t)c2 * (2 * slot_floats / 4) + (size_t)q * TM) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 acc = t[0][q];
+#pragma unroll
+            for (int c2 = 1; c2 < 4; ++c2) { acc.x += t[c2][q].x; acc.y += t[c2][q].y; acc.z += t[c2][q].z; acc.w += t[c2][q].w; }
+            v[4 * q] = __float_as_uint(acc.x); v[4 * q + 1] = __float_as_uint(acc.y);
+            v[4 * q + 2] = __float_as_uint(acc.z); v[4 * q + 3] = __float_as_uint(acc.w);
+          }
+        }
+      };
       if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < (OUT_COLS / 32); ++c) {
           uint32_t v[32];
-          tmem_ld32(tbase + c * 32, v);
-          tmem_ld_wait();
+          load_chunk(c * 32, v);
           const int col0 = n0 + c * 32;
           if (!row_ok || col0 >= g.N) continue;
           bf16* dst = g.C + (size_t)row * g.ldc + col0;
@@ -314,9 +383,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll 1
         for (int c = 0; c < (OUT_COLS / 32); ++c) {
           uint32_t gv[32], uv[32];
-          tmem_ld32(tbase + c * 32, gv);
-          tmem_ld32(tbase + 128 + c * 32, uv);
-          tmem_ld_wait();
+          load_chunk(c * 32, gv);
+          load_chunk(128 + c * 32, uv);
           const int col0 = n0 + c * 32;
           if (!row_ok || col0 >= g.N) continue;
           bf16* dst = g.C + (size_t)row * g.ldc + col0;
@@ -349,8 +417,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             uint32_t v[32];
-            tmem_ld32(tbase + half * 128 + c * 32, v);
-            tmem_ld_wait();
+            load_chunk(half * 128 + c * 32, v);
             const int col0 = n0 + half * 128 + c * 32;
             if (col0 >= g.N) continue;
             float cmx = -INFINITY; int carg = 0x7fffffff;
@@ -381,10 +448,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
       }
-      // hand the accumulator back to the MMA thread in the even CTA
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_even_cta(acc_empty(buf));
+      // hand the accumulator back to the MMA thread in the even CTA (a split-K part has done so already)
+      if (!reduce) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_even_cta(acc_empty(buf));
+      }
     }
   }
   // ------------------------------------------------------------------ teardown
