@@ -22,7 +22,6 @@ namespace {
 constexpr int AQ = 128, AKEYS = 128, ADH = 128;
 constexpr int HALF_BYTES = 128 * 64 * 2;          // one 128-row x 64-column swizzled box: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;        // 128 x 128 bf16
-constexpr int ATC_THREADS = 192;
 constexpr long long kWaitCycles = 4000000000LL;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 

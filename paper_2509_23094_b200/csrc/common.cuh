@@ -85,7 +85,7 @@ int launch_rope_scatter(bf16* qkv, const int32_t* sel_idx, const int32_t* row_se
                         int cache_seq, cudaStream_t st);
 
 // ---- GEMMs (gemm_mma.cu, gemm_tc.cu) -----------------------------------------------------------
-enum GemmEpilogue { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_LMSTATS = 3 };
+enum GemmEpilogue { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_LMSTATS = 3, EPI_QKV_ROPE = 4 };
 struct GemmArgs {
   const bf16* A; int lda;            // [max_rows][K]
   const bf16* W; const bf16* W2;     // [N][K]; W2 = the "up" matrix for EPI_SWIGLU
@@ -94,6 +94,10 @@ struct GemmArgs {
   const int32_t* n_rows; int max_rows; int N; int K;
   // EPI_LMSTATS: per (row, 128-column tile) running max / sum of exp / arg-max, optional raw logits
   float* st_max; float* st_sum; int32_t* st_arg; float* logits; int n_tiles;
+  // EPI_QKV_ROPE (tcgen05 kernels only): rotary embedding of Q/K and the K/V scatter into the cache fused into
+  // the QKV projection; C/ldc is the QKV activation buffer (only its Q part is written)
+  const int32_t* q_sel_idx; const int32_t* q_row_seq; const float2* q_rope; bf16* q_kc; bf16* q_vc;
+  int q_cache_seq, q_hq, q_hkv, q_dh;
   // split-K scratch of the one-SM tcgen05 kernel (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
   // and as many zero-initialised arrival counters
   float* sk_partials; int32_t* sk_counters; int sk_max_tiles;
@@ -141,6 +145,7 @@ int launch_commit(int batch, int seq_len, int d, int rule, float threshold, cons
 // ---- tcgen05 GEMM (gemm_tc.cu) -------------------------------------------------------------------
 // status: device int[4] that receives D2C_ETIMEOUT if a bounded wait runs out (null: a library-owned word).
 int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status = nullptr);
+bool gemm_tc_supported(const GemmArgs& g);       // false: launch_gemm_tc would fall back to the mma.sync kernel
 // ---- two-SM tcgen05 GEMM (gemm_tc2.cu): pairs of CTAs on 256-row tiles ---------------------------
 bool gemm_tc2_supported(const GemmArgs& g);
 int launch_gemm_tc2(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status = nullptr);

@@ -313,10 +313,17 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     GemmArgs g{};
     g.A = b.xn; g.lda = d; g.W = ctx->wqkv[l]; g.bias = ctx->bqkv[l]; g.C = b.qkv; g.ldc = qkv_out;
     g.n_rows = n_rows; g.max_rows = R; g.N = qkv_out; g.K = d;
-    D2C_TRY(ctx, gemm(ctx, g, EPI_STORE));
     bf16* kc = b.kcache + (size_t)l * cache_layer; bf16* vc = b.vcache + (size_t)l * cache_layer;
-    D2C_TRY(ctx, mark(ctx, PH_ROPE));
-    D2C_TRY(ctx, launch_rope_scatter(b.qkv, b.sel_idx, b.row_seq, n_rows, R, hq, hkv, dh, b.rope, kc, vc, c.max_seq, st));
+    if (!(c.flags & D2C_FLAG_PORTABLE_GEMM) && gemm_tc_supported(g)) {
+      // QKV projection with bias, rotary embedding and the K/V scatter in its epilogue
+      g.q_sel_idx = b.sel_idx; g.q_row_seq = b.row_seq; g.q_rope = b.rope; g.q_kc = kc; g.q_vc = vc;
+      g.q_cache_seq = c.max_seq; g.q_hq = hq; g.q_hkv = hkv; g.q_dh = dh;
+      D2C_TRY(ctx, gemm(ctx, g, EPI_QKV_ROPE));
+    } else {
+      D2C_TRY(ctx, gemm(ctx, g, EPI_STORE));
+      D2C_TRY(ctx, mark(ctx, PH_ROPE));
+      D2C_TRY(ctx, launch_rope_scatter(b.qkv, b.sel_idx, b.row_seq, n_rows, R, hq, hkv, dh, b.rope, kc, vc, c.max_seq, st));
+    }
     AttnArgs at{};
     at.q = b.qkv; at.ldq = qkv_out; at.kc = kc; at.vc = vc; at.row_off = b.row_off; at.batch = B; at.seq_len = L;
     at.cache_seq = c.max_seq; at.hq = hq; at.hkv = hkv; at.dh = dh; at.max_rows_per_seq = L;

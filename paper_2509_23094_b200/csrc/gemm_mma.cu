@@ -244,6 +244,7 @@ int launch_gemm_mma(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st) {
     case EPI_RESIDUAL: return launch_one<EPI_RESIDUAL>(g, st);
     case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(g, st);
     case EPI_LMSTATS: return launch_one<EPI_LMSTATS>(g, st);
+    default: break;
   }
   return D2C_EINVAL;
 }

@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "epilogue_qkv.cuh"
 
 namespace d2c {
 namespace {
@@ -141,7 +142,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   // Accumulator width of this launch: 256 columns, narrowed to 128 or 64 while that still leaves SMs
   // without a tile (few live rows and a small N), so that more SMs stream the weights.
   int bn = ACC_COLS;
-  const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : 64);
+  const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? max(64, g.q_dh) : 64));
   while (bn > bn_min && 2 * MT * ((g.N + bn - 1) / bn) <= (int)gridDim.x) bn >>= 1;
   const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
@@ -327,7 +328,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
           }
         }
       };
-      if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+      if (EPI == EPI_QKV_ROPE) {
+        epilogue_qkv_rope(load_chunk, g, row, row_ok, n0, OUT_COLS);
+      } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < n_chunks; ++c) {
@@ -511,7 +514,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   if (rc == D2C_OK) rc = make_map(&tmB64, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 64);
   if (rc != D2C_OK) return rc;
   TcParams p{g, status};
-  const int out_cols = EPI == EPI_SWIGLU ? 128 : (EPI == EPI_LMSTATS ? 128 : 64);   // narrowest tile the kernel may pick
+  const int out_cols = EPI == EPI_SWIGLU ? 128 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? (g.q_dh > 64 ? g.q_dh : 64) : 64));   // narrowest tile
   const long long tiles = (long long)ceil_div(g.max_rows, TM) * ceil_div(g.N, out_cols);
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
   D2C_LAUNCH((gemm_tc_kernel<EPI>), grid, TC_THREADS, smem, st, tmA128, tmA64, tmA32, tmB, tmB2, tmB64, p);
@@ -519,17 +522,24 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
 }
 }  // namespace
 
+bool gemm_tc_supported(const GemmArgs& g) {
+  return !(g.max_rows < TM || g.N < 128 || g.K % TK != 0 || (g.lda & 7) || (g.N & 1) ||
+           (reinterpret_cast<uintptr_t>(g.A) & 15) || (reinterpret_cast<uintptr_t>(g.W) & 15));
+}
+
 int launch_gemm_tc(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* status) {
   if (g.max_rows <= 0 || g.N <= 0) return D2C_OK;
   // shapes the TMA boxes cannot express fall back to the portable kernel
-  if (g.max_rows < TM || g.N < 128 || g.K % TK != 0 || (g.lda & 7) || (g.N & 1) ||
-      (reinterpret_cast<uintptr_t>(g.A) & 15) || (reinterpret_cast<uintptr_t>(g.W) & 15))
+  if (!gemm_tc_supported(g)) {
+    if (epi == EPI_QKV_ROPE) { set_global_error("gemm: the fused QKV epilogue needs the tcgen05 kernel"); return D2C_ESHAPE; }
     return launch_gemm_mma(g, epi, st);
+  }
   switch (epi) {
     case EPI_STORE: return launch_one<EPI_STORE>(g, status, st);
     case EPI_RESIDUAL: return launch_one<EPI_RESIDUAL>(g, status, st);
     case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(g, status, st);
     case EPI_LMSTATS: return launch_one<EPI_LMSTATS>(g, status, st);
+    case EPI_QKV_ROPE: return launch_one<EPI_QKV_ROPE>(g, status, st);
   }
   return D2C_EINVAL;
 }

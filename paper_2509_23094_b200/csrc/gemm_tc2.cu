@@ -12,6 +12,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "epilogue_qkv.cuh"
 
 namespace d2c {
 namespace {
@@ -57,28 +58,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
                "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -100,10 +81,6 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   d |= (uint64_t)1 << 46;                        // descriptor version of sm_100
   d |= (uint64_t)2 << 61;                        // 128-byte swizzle
   return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
 }
 
 union Pack8 { uint4 u; __nv_bfloat162 h[4]; };
@@ -340,7 +317,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
       };
-      if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+      if (EPI == EPI_QKV_ROPE) {
+        epilogue_qkv_rope(load_chunk, g, row, row_ok, n0, OUT_COLS);
+      } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < (OUT_COLS / 32); ++c) {
@@ -525,7 +504,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   if (rc == D2C_OK) rc = make_map(&tmB32, g.W, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.K, 32);
   if (rc != D2C_OK) return rc;
   Tc2Params p{g, status};
-  const int out_cols = (EPI == EPI_STORE || EPI == EPI_RESIDUAL) ? 64 : (EPI == EPI_SWIGLU ? 128 : 256);   // narrowest tile
+  const int out_cols = (EPI == EPI_STORE || EPI == EPI_RESIDUAL) ? 64 : (EPI == EPI_SWIGLU ? 128 : 256);   // narrowest tile (QKV: 256)
   const long long tiles = (long long)ceil_div(g.max_rows, 2 * TM) * ceil_div(g.N, out_cols);
   const int pairs = (int)(tiles < sm_count2() / 2 ? tiles : sm_count2() / 2);
   cudaLaunchConfig_t cfg = {};
@@ -554,6 +533,7 @@ int launch_gemm_tc2(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st, int* s
     case EPI_RESIDUAL: return launch_one<EPI_RESIDUAL>(g, status, st);
     case EPI_SWIGLU: return launch_one<EPI_SWIGLU>(g, status, st);
     case EPI_LMSTATS: return launch_one<EPI_LMSTATS>(g, status, st);
+    case EPI_QKV_ROPE: return launch_one<EPI_QKV_ROPE>(g, status, st);
   }
   return D2C_EINVAL;
 }
