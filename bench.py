@@ -222,7 +222,7 @@ def run_ours(args, rank, world, device):
         if i >= 2:
             e2e_s += time.perf_counter() - t0
     h2d = B * L * d * 2 + B * L
-    d2h = (B + 1) * 4 + n * 4 + n * d * 2 + 2 * B * L * 4
+    d2h = (B + 1) * 4 + B * L * 4 + B * L * d * 2 + 2 * B * L * 4       # worst-case sizes: the row count is not known when the copies start
 
     total_ms, e2e_s, n_all = aggregate_replicas(total_ms, e2e_s, float(n), world, device)
     ms_per_step = total_ms / args.steps

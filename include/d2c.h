@@ -133,7 +133,8 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* args, const d2c_step_out* out);
 /* The same step for callers whose data lives in HOST memory: h0, mask, forced,
  * forced_off and the override vectors are host pointers (pinned memory makes
  * the copies asynchronous); the outputs are host buffers: sel_idx_host
- * [max rows], row_off_host [batch+1], hidden_out_host bf16 [max rows][d],
+ * [batch*seq_len], row_off_host [batch+1], hidden_out_host bf16 [batch*seq_len][d] (the copy starts before the row
+ * count is known, so the whole buffer may be written; rows beyond row_off_host[batch] are meaningless),
  * conf_host / pred_host [batch][seq_len] (any may be NULL).  Copies in, runs
  * d2c_step, copies out, and synchronises the stream before returning. */
 typedef struct {

@@ -117,6 +117,11 @@ struct d2c_ctx {
   // Selected-row count of an earlier step, copied to pinned host memory at the end of every step and read
   // without synchronising: only a hint for choosing between GEMM kernels (both are correct for any count).
   int32_t* n_hint = nullptr;
+  // d2c_step_host: the device-to-host copy of the hidden rows runs on its own stream, ordered after the
+  // last layer by an event, so that it overlaps the LM head and the rollout
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t layers_done = nullptr;
+  void* early_hidden_host = nullptr;     // set by d2c_step_host for the duration of one step
   char err[512];
   // optional per-phase timing: one event at every phase boundary, resolved by d2c_profile_read
   bool prof = false;
@@ -213,6 +218,11 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
   carve(*cfg, workspace, &ctx->buf);
   if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->n_hint), sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess) *ctx->n_hint = 1 << 30;
   else { ctx->n_hint = nullptr; (void)cudaGetLastError(); }
+  if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->layers_done, cudaEventDisableTiming) != cudaSuccess) {
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    ctx->copy_stream = nullptr; ctx->layers_done = nullptr; (void)cudaGetLastError();
+  }
   cudaError_t e = cudaMemsetAsync(workspace, 0, need, ctx->stream);
   if (e == cudaSuccess) {
     std::vector<uint32_t> tab(cfg->max_seq);
@@ -233,6 +243,8 @@ int d2c_destroy(d2c_ctx* ctx) {
   if (!ctx) return D2C_EINVAL;
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   if (ctx->n_hint) cudaFreeHost(ctx->n_hint);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->layers_done) cudaEventDestroy(ctx->layers_done);
   delete ctx;
   return D2C_OK;
 }
@@ -354,6 +366,14 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     D2C_TRY(ctx, mark(ctx, PH_DOWN));
     D2C_TRY(ctx, gemm(ctx, gd, EPI_RESIDUAL));
   }
+  if (ctx->early_hidden_host && ctx->copy_stream) {
+    // the residual stream is final here: ship it to the host while the LM head and the rollout run
+    // (the row count is not known on the host yet, so the worst case is copied)
+    cudaError_t e = cudaEventRecord(ctx->layers_done, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->layers_done, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->early_hidden_host, x, (size_t)R * d * sizeof(bf16), cudaMemcpyDeviceToHost, ctx->copy_stream);
+    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
+  }
   // Eq. 1 on the selected rows that are still masked
   D2C_TRY(ctx, mark(ctx, PH_LM));
   D2C_TRY(ctx, launch_rmsnorm(x, b.lm_rows, n_lm, R, d, ctx->g_final, c.rms_eps, b.xm, st));
@@ -438,25 +458,22 @@ int d2c_step_host(d2c_ctx* ctx, const d2c_step_args* h, const d2c_host_out* out)
   if (h->override_key) { D2C_CP(b.okey_stage, h->override_key, R * sizeof(float), cudaMemcpyHostToDevice); a.override_key = b.okey_stage; }
   if (h->override_c) { D2C_CP(b.oc_stage, h->override_c, R * sizeof(float), cudaMemcpyHostToDevice); a.override_c = b.oc_stage; }
   d2c_step_out dev_out{};
-  D2C_TRY(ctx, d2c_step(ctx, &a, &dev_out));
-  std::vector<int32_t> ro(B + 1);
-  D2C_CP(ro.data(), b.row_off, (B + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost);
-  cudaError_t e = cudaStreamSynchronize(st);
-  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e));
-  const size_t n = (size_t)ro[B];
+  const bool early = out && out->hidden_out_host && ctx->copy_stream;
+  ctx->early_hidden_host = early ? out->hidden_out_host : nullptr;
+  const int step_rc = d2c_step(ctx, &a, &dev_out);
+  ctx->early_hidden_host = nullptr;
+  if (step_rc != D2C_OK) { if (early) cudaStreamSynchronize(ctx->copy_stream); return step_rc; }
+  // every result is copied without knowing the row count (worst-case sizes), then one synchronisation
   if (out) {
-    if (out->row_off_host) memcpy(out->row_off_host, ro.data(), (B + 1) * sizeof(int32_t));
-    if (out->sel_idx_host && n) D2C_CP(out->sel_idx_host, b.sel_idx, n * sizeof(int32_t), cudaMemcpyDeviceToHost);
-    if (out->hidden_out_host && n) D2C_CP(out->hidden_out_host, b.x, n * c.d_model * sizeof(bf16), cudaMemcpyDeviceToHost);
-    if (out->conf_host) {
-      for (size_t bb = 0; bb < B; ++bb) D2C_CP(out->conf_host + bb * L, b.conf + bb * L, L * sizeof(float), cudaMemcpyDeviceToHost);
-    }
-    if (out->pred_host) {
-      for (size_t bb = 0; bb < B; ++bb) D2C_CP(out->pred_host + bb * L, b.pred + bb * L, L * sizeof(int32_t), cudaMemcpyDeviceToHost);
-    }
-    e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e));
+    if (out->row_off_host) D2C_CP(out->row_off_host, b.row_off, (B + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    if (out->sel_idx_host) D2C_CP(out->sel_idx_host, b.sel_idx, R * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    if (out->hidden_out_host && !early) D2C_CP(out->hidden_out_host, b.x, R * c.d_model * sizeof(bf16), cudaMemcpyDeviceToHost);
+    if (out->conf_host) D2C_CP(out->conf_host, b.conf, R * sizeof(float), cudaMemcpyDeviceToHost);
+    if (out->pred_host) D2C_CP(out->pred_host, b.pred, R * sizeof(int32_t), cudaMemcpyDeviceToHost);
   }
+  cudaError_t e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess && early) e = cudaStreamSynchronize(ctx->copy_stream);
+  if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step_host: %s", cudaGetErrorString(e));
 #undef D2C_CP
   return D2C_OK;
 }
