@@ -233,7 +233,7 @@ def run_ours(args, rank, world, device):
     depth = shape.n_layers
     flops, byts = algorithmic_work(shape, B, L, n_b, n_m, depth)
     t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
-    # dominant kernel: the gate/up projection GEMM (gemm_tc_kernel<EPI_SWIGLU>, one launch per layer); its
+    # dominant kernel: the gate/up projection GEMM (gemm_tc2_kernel<EPI_SWIGLU>, one launch per layer); its
     # average launch duration comes from the events of the second timed pass
     gu_ms = phases["gemm_gate_up"]["ms"] / args.steps / shape.n_layers
     gu_flops = 2 * n * d * 2 * shape.d_ffn
@@ -241,8 +241,8 @@ def run_ours(args, rank, world, device):
     gemm_ms = sum(phases[k]["ms"] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) / args.steps
     gemm_flops = shape.n_layers * 2 * n * shape.params_per_layer
     # DRAM bytes of one launch from the committed ncu capture of this workload (profiles/), null elsewhere
-    traffic = 224.7e6 if wl.name == "llada1l_1024" else None
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel<SWIGLU> (gate/up projection, 1 launch per layer)",
+    traffic = 229.4e6 if wl.name == "llada1l_1024" else None
+    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel<SWIGLU> (gate/up projection, 1 launch per layer)",
                 "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst",
                 "unit": "TFLOP/s", "frac": round(achieved / peaks["bf16_tflops"], 4), "traffic": traffic,
                 "algorithmic_bytes": 2 * d * 2 * shape.d_ffn + n * d * 2 + n * shape.d_ffn * 2,
