@@ -62,6 +62,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
 }
@@ -134,29 +137,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant__ CUtensorMap tmA64,
                const __grid_constant__ CUtensorMap tmA32, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmB64, const TcParams p) {
-  pdl_prologue();
+  // Everything that does not read a predecessor's results (barriers, TMEM, descriptor prefetch) runs before
+  // the wait on the preceding kernel, so it overlaps that kernel's tail.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const GemmArgs& g = p.g;
-  const int n = *g.n_rows;
-  if (n <= 0) return;
-  const int MT = (n + TM - 1) / TM;
-  // Accumulator width of this launch: 256 columns, narrowed to 128 or 64 while that still leaves SMs
-  // without a tile (few live rows and a small N), so that more SMs stream the weights.
-  int bn = ACC_COLS;
-  const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? max(64, g.q_dh) : 64));
-  while (bn > bn_min && 2 * MT * ((g.N + bn - 1) / bn) <= (int)gridDim.x) bn >>= 1;
-  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
-  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
-  const int total = MT * NT;
-  const int KT = g.K / TK, G = gridDim.x;
-  // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
-  // idle SM is lost bandwidth): each tile's K range is cut into S equal parts handled by different CTAs.
-  // Parts park their fp32 accumulators in scratch; the part that arrives last adds them in part order
-  // (no waiting, deterministic) and runs the epilogue.
-  int S = 1;
-  if (g.sk_partials != nullptr && g.sk_counters != nullptr && total < G && total <= g.sk_max_tiles)
-    S = max(1, min(min(G / total, KT / 8), 4));
-  const int items = total * S;
-  if ((int)blockIdx.x >= items) return;                      // uniform: nothing allocated yet
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int* status = p.status ? p.status : g_tc_status;
 
@@ -170,19 +154,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   auto empty_bar = [&](int s) { return bar0 + 8u * (ST_MAX + s); };
   auto acc_full = [&](int b) { return bar0 + 8u * (2 * ST_MAX + b); };
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * ST_MAX + 2 + b); };
-  // Stage size follows the tile this launch uses (A box of 128 rows or less, bn weight rows); the freed
-  // shared memory becomes more stages, i.e. more bytes in flight per SM when the launch streams weights.
-  const int a_rows_max = n >= 128 ? 128 : (n > 64 ? 128 : (n > 32 ? 64 : 32));
-  const int stage_bytes = ((a_rows_max + ((EPI == EPI_SWIGLU) ? ACC_COLS : bn)) * TK * 2 + 1023) & ~1023;
-  // the MMA always reads 128 rows of A: keep that read inside the allocation when the A box is smaller
-  const int nst = min(ST_MAX, (ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2) / stage_bytes);
-
   if (threadIdx.x == 0) {
-    for (int s = 0; s < nst; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < ST_MAX; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    prefetch_tensormap(&tmA128); prefetch_tensormap(&tmB); prefetch_tensormap(&tmB2);
   }
   if (warp == 1) {
     tmem_alloc((uint32_t)__cvta_generic_to_shared(&tmem_slot), 2 * ACC_COLS);
@@ -193,6 +171,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_acc = tmem_slot;
   volatile int* abortp = &abort_flag;
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int n = max(*g.n_rows, 0);
+  const int MT = (n + TM - 1) / TM;
+  // Accumulator width of this launch: 256 columns, narrowed to 128 or 64 while that still leaves SMs
+  // without a tile (few live rows and a small N), so that more SMs stream the weights.
+  int bn = ACC_COLS;
+  const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? max(64, g.q_dh) : 64));
+  while (bn > bn_min && 2 * MT * ((g.N + bn - 1) / bn) <= (int)gridDim.x) bn >>= 1;
+  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
+  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int total = MT * NT;                                 // 0 when no row is live: every role loop is empty
+  const int KT = g.K / TK, G = gridDim.x;
+  // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
+  // idle SM is lost bandwidth): each tile's K range is cut into S equal parts handled by different CTAs.
+  // Parts park their fp32 accumulators in scratch; the part that arrives last adds them in part order
+  // (no waiting, deterministic) and runs the epilogue.
+  int S = 1;
+  if (g.sk_partials != nullptr && g.sk_counters != nullptr && total > 0 && total < G && total <= g.sk_max_tiles)
+    S = max(1, min(min(G / total, KT / 8), 4));
+  const int items = total * S;
+  // Stage size follows the tile this launch uses (A box of 128 rows or less, bn weight rows); the freed
+  // shared memory becomes more stages, i.e. more bytes in flight per SM when the launch streams weights.
+  const int a_rows_max = n >= 128 ? 128 : (n > 64 ? 128 : (n > 32 ? 64 : 32));
+  const int stage_bytes = ((a_rows_max + ((EPI == EPI_SWIGLU) ? ACC_COLS : bn)) * TK * 2 + 1023) & ~1023;
+  // the MMA always reads 128 rows of A: keep that read inside the allocation when the A box is smaller
+  const int nst = min(ST_MAX, (ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2) / stage_bytes);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -270,6 +275,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       const int n_chunks = OUT_COLS / 32;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
+      const bool vec = (g.ldc & 7) == 0;
+      // The residual is read two chunks ahead of the accumulator (the first two before the accumulator is
+      // complete) so that its latency is hidden.
+      uint4 r0[4], r1[4], r2[4];
+      auto load_res = [&](int c, uint4 (&r)[4]) {
+        const int col0 = n0 + c * 32;
+        if (EPI == EPI_RESIDUAL && row_ok && vec && c < n_chunks && col0 + 32 <= g.N) {
+          const uint4* src = reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) r[q] = __ldcg(src + q);
+        }
+      };
+      load_res(0, r0); load_res(1, r1);
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 3)) break;
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
@@ -331,43 +349,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       if (EPI == EPI_QKV_ROPE) {
         epilogue_qkv_rope(load_chunk, g, row, row_ok, n0, OUT_COLS);
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-        const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < n_chunks; ++c) {
           uint32_t v[32];
+          load_res(c + 2, r2);
           load_chunk(c * 32, v);
           const int col0 = n0 + c * 32;
-          if (!row_ok || col0 >= g.N) continue;
-          bf16* dst = g.C + (size_t)row * g.ldc + col0;
-          if (vec && col0 + 32 <= g.N) {
+          if (row_ok && col0 < g.N) {
+            bf16* dst = g.C + (size_t)row * g.ldc + col0;
+            if (vec && col0 + 32 <= g.N) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              Pack8 o, old;
-              if (EPI == EPI_RESIDUAL) old.u = reinterpret_cast<const uint4*>(dst)[q];
+              for (int q = 0; q < 4; ++q) {
+                Pack8 o, old;
+                if (EPI == EPI_RESIDUAL) old.u = r0[q];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
-                if (EPI == EPI_STORE) {
-                  if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
-                } else {
-                  const float2 of = __bfloat1622float2(old.h[e]);
-                  f0 += of.x; f1 += of.y;
+                for (int e = 0; e < 4; ++e) {
+                  float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
+                  if (EPI == EPI_STORE) {
+                    if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
+                  } else {
+                    const float2 of = __bfloat1622float2(old.h[e]);
+                    f0 += of.x; f1 += of.y;
+                  }
+                  o.h[e] = __floats2bfloat162_rn(f0, f1);
                 }
-                o.h[e] = __floats2bfloat162_rn(f0, f1);
+                reinterpret_cast<uint4*>(dst)[q] = o.u;
               }
-              reinterpret_cast<uint4*>(dst)[q] = o.u;
-            }
-          } else {
+            } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (col0 + j < g.N) {
-                float f = __uint_as_float(v[j]);
-                if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
-                else f += __bfloat162float(dst[j]);
-                dst[j] = __float2bfloat16_rn(f);
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j < g.N) {
+                  float f = __uint_as_float(v[j]);
+                  if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
+                  else f += __bfloat162float(dst[j]);
+                  dst[j] = __float2bfloat16_rn(f);
+                }
               }
             }
           }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { r0[q] = r1[q]; r1[q] = r2[q]; }
         }
       } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1

@@ -96,6 +96,9 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
   asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar & kPeerMask), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc2(uint32_t slot, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
 }
@@ -125,38 +128,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmB64,
                 const __grid_constant__ CUtensorMap tmB32, const Tc2Params p) {
-  pdl_prologue();
+  // Everything that does not read a predecessor's results (barriers, TMEM, descriptor prefetch) runs before
+  // the wait on the preceding kernel, so it overlaps that kernel's tail.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const GemmArgs& g = p.g;
-  const int n = *g.n_rows;
-  if (n <= 0) return;
-  const int MT = (n + 2 * TM - 1) / (2 * TM);
   const int cl = blockIdx.x >> 1, ncl = gridDim.x >> 1;
-  // Accumulator width: 256 columns, halved (to 128, then 64) while the narrower tiling fills the last
-  // wave of clusters so much better that it outweighs the far less efficient narrow MMA (measured factor ~0.6).
-  int bn = ACC_COLS;
-  const int KT = g.K / TK;
-  const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
-  const int t256 = MT * ((g.N + (EPI == EPI_SWIGLU ? 128 : 256) - 1) / (EPI == EPI_SWIGLU ? 128 : 256));
-  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;   // split-K beats narrow tiles
-  if ((EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split) {
-    while (bn > 64) {
-      const int t_wide = MT * ((g.N + bn - 1) / bn), t_narrow = MT * ((g.N + bn / 2 - 1) / (bn / 2));
-      const float e_wide = (float)t_wide / (float)(((t_wide + ncl - 1) / ncl) * ncl);
-      const float e_narrow = (float)t_narrow / (float)(((t_narrow + ncl - 1) / ncl) * ncl);
-      if (e_narrow * 0.6f > e_wide) bn >>= 1; else break;
-    }
-  }
-  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per pair-tile
-  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
-  const int total = MT * NT;
-  // Split-K when there are fewer pair-tiles than clusters: K is cut into S equal parts, one (tile, part)
-  // item per cluster; every CTA parks its 128 rows of fp32 partial sums in scratch and, per (tile, CTA
-  // rank), the part that arrives last adds all parts in part order (no waiting, deterministic).
-  int S = 1;
-  if (sk_ok && total < ncl && 2 * total <= g.sk_max_tiles)
-    S = max(1, min(min(ncl / total, KT / 8), 4));
-  const int items = total * S;
-  if (cl >= items) return;                                   // same answer in both CTAs of a cluster
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -179,6 +155,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    prefetch_tensormap(&tmA); prefetch_tensormap(&tmB); prefetch_tensormap(&tmB2);
   }
   if (warp == 1) {
     tmem_alloc2((uint32_t)__cvta_generic_to_shared(&tmem_slot), 2 * ACC_COLS);
@@ -190,6 +167,36 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_acc = tmem_slot;
   volatile int* abortp = &abort_flag;
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int n = *g.n_rows;
+  const int MT = (max(n, 0) + 2 * TM - 1) / (2 * TM);
+  // Accumulator width: 256 columns, halved (to 128, then 64) while the narrower tiling fills the last
+  // wave of clusters so much better that it outweighs the far less efficient narrow MMA (measured factor ~0.6).
+  int bn = ACC_COLS;
+  const int KT = g.K / TK;
+  const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
+  const int t256 = MT * ((g.N + (EPI == EPI_SWIGLU ? 128 : 256) - 1) / (EPI == EPI_SWIGLU ? 128 : 256));
+  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;   // split-K beats narrow tiles
+  if ((EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split) {
+    while (bn > 64) {
+      const int t_wide = MT * ((g.N + bn - 1) / bn), t_narrow = MT * ((g.N + bn / 2 - 1) / (bn / 2));
+      if (t_wide == 0) break;
+      const float e_wide = (float)t_wide / (float)(((t_wide + ncl - 1) / ncl) * ncl);
+      const float e_narrow = (float)t_narrow / (float)(((t_narrow + ncl - 1) / ncl) * ncl);
+      if (e_narrow * 0.6f > e_wide) bn >>= 1; else break;
+    }
+  }
+  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per pair-tile
+  const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
+  const int total = MT * NT;                                 // 0 when no row is live: every role loop is empty
+  // Split-K when there are fewer pair-tiles than clusters: K is cut into S equal parts, one (tile, part)
+  // item per cluster; every CTA parks its 128 rows of fp32 partial sums in scratch and, per (tile, CTA
+  // rank), the part that arrives last adds all parts in part order (no waiting, deterministic).
+  int S = 1;
+  if (sk_ok && total > 0 && total < ncl && 2 * total <= g.sk_max_tiles)
+    S = max(1, min(min(ncl / total, KT / 8), 4));
+  const int items = total * S;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -258,6 +265,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
+      const bool vec = (g.ldc & 7) == 0;
+      // The residual is read two chunks ahead of the accumulator (the first two before the accumulator is
+      // complete) so that its latency is hidden.
+      uint4 r0[4], r1[4], r2[4];
+      auto load_res = [&](int c, uint4 (&r)[4]) {
+        const int col0 = n0 + c * 32;
+        if (EPI == EPI_RESIDUAL && row_ok && vec && c < OUT_COLS / 32 && col0 + 32 <= g.N) {
+          const uint4* src = reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) r[q] = __ldcg(src + q);
+        }
+      };
+      load_res(0, r0); load_res(1, r1);
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 33)) break;
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
@@ -320,43 +340,46 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (EPI == EPI_QKV_ROPE) {
         epilogue_qkv_rope(load_chunk, g, row, row_ok, n0, OUT_COLS);
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-        const bool vec = (g.ldc & 7) == 0;
 #pragma unroll 1
         for (int c = 0; c < (OUT_COLS / 32); ++c) {
           uint32_t v[32];
+          load_res(c + 2, r2);
           load_chunk(c * 32, v);
           const int col0 = n0 + c * 32;
-          if (!row_ok || col0 >= g.N) continue;
-          bf16* dst = g.C + (size_t)row * g.ldc + col0;
-          if (vec && col0 + 32 <= g.N) {
+          if (row_ok && col0 < g.N) {
+            bf16* dst = g.C + (size_t)row * g.ldc + col0;
+            if (vec && col0 + 32 <= g.N) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              Pack8 o, old;
-              if (EPI == EPI_RESIDUAL) old.u = reinterpret_cast<const uint4*>(dst)[q];
+              for (int q = 0; q < 4; ++q) {
+                Pack8 o, old;
+                if (EPI == EPI_RESIDUAL) old.u = r0[q];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
-                if (EPI == EPI_STORE) {
-                  if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
-                } else {
-                  const float2 of = __bfloat1622float2(old.h[e]);
-                  f0 += of.x; f1 += of.y;
+                for (int e = 0; e < 4; ++e) {
+                  float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
+                  if (EPI == EPI_STORE) {
+                    if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
+                  } else {
+                    const float2 of = __bfloat1622float2(old.h[e]);
+                    f0 += of.x; f1 += of.y;
+                  }
+                  o.h[e] = __floats2bfloat162_rn(f0, f1);
                 }
-                o.h[e] = __floats2bfloat162_rn(f0, f1);
+                reinterpret_cast<uint4*>(dst)[q] = o.u;
               }
-              reinterpret_cast<uint4*>(dst)[q] = o.u;
-            }
-          } else {
+            } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (col0 + j < g.N) {
-                float f = __uint_as_float(v[j]);
-                if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
-                else f += __bfloat162float(dst[j]);
-                dst[j] = __float2bfloat16_rn(f);
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j < g.N) {
+                  float f = __uint_as_float(v[j]);
+                  if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
+                  else f += __bfloat162float(dst[j]);
+                  dst[j] = __float2bfloat16_rn(f);
+                }
               }
             }
           }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { r0[q] = r1[q]; r1[q] = r2[q]; }
         }
       } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
