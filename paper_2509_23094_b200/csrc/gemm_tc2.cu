@@ -12,7 +12,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
-#include "epilogue_qkv.cuh"
+#include "epilogue_tiles.cuh"
 
 namespace d2c {
 namespace {
@@ -265,19 +265,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
-      const bool vec = (g.ldc & 7) == 0;
-      // The residual is read two chunks ahead of the accumulator (the first two before the accumulator is
-      // complete) so that its latency is hidden.
-      uint4 r0[4], r1[4], r2[4];
-      auto load_res = [&](int c, uint4 (&r)[4]) {
-        const int col0 = n0 + c * 32;
-        if (EPI == EPI_RESIDUAL && row_ok && vec && c < OUT_COLS / 32 && col0 + 32 <= g.N) {
-          const uint4* src = reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col0);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) r[q] = __ldcg(src + q);
-        }
-      };
-      load_res(0, r0); load_res(1, r1);
       if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 33)) break;
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
@@ -337,81 +324,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
       };
+      const EpiWarp ew{smem_base + (uint32_t)(ST2 * STAGE2) + (uint32_t)(quarter * kEpiStageBytes), m0 + quarter * 32, n, lane};
       if (EPI == EPI_QKV_ROPE) {
-        epilogue_qkv_rope(load_chunk, g, row, row_ok, n0, OUT_COLS);
+        epilogue_qkv_rope(load_chunk, g, ew, n0, OUT_COLS);
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-#pragma unroll 1
-        for (int c = 0; c < (OUT_COLS / 32); ++c) {
-          uint32_t v[32];
-          load_res(c + 2, r2);
-          load_chunk(c * 32, v);
-          const int col0 = n0 + c * 32;
-          if (row_ok && col0 < g.N) {
-            bf16* dst = g.C + (size_t)row * g.ldc + col0;
-            if (vec && col0 + 32 <= g.N) {
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                Pack8 o, old;
-                if (EPI == EPI_RESIDUAL) old.u = r0[q];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  float f0 = __uint_as_float(v[q * 8 + 2 * e]), f1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
-                  if (EPI == EPI_STORE) {
-                    if (g.bias) { f0 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e]); f1 += __bfloat162float(g.bias[col0 + q * 8 + 2 * e + 1]); }
-                  } else {
-                    const float2 of = __bfloat1622float2(old.h[e]);
-                    f0 += of.x; f1 += of.y;
-                  }
-                  o.h[e] = __floats2bfloat162_rn(f0, f1);
-                }
-                reinterpret_cast<uint4*>(dst)[q] = o.u;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (col0 + j < g.N) {
-                  float f = __uint_as_float(v[j]);
-                  if (EPI == EPI_STORE) { if (g.bias) f += __bfloat162float(g.bias[col0 + j]); }
-                  else f += __bfloat162float(dst[j]);
-                  dst[j] = __float2bfloat16_rn(f);
-                }
-              }
-            }
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) { r0[q] = r1[q]; r1[q] = r2[q]; }
-        }
+        epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS);
       } else if (EPI == EPI_SWIGLU) {
-#pragma unroll 1
-        for (int c = 0; c < (OUT_COLS / 32); ++c) {
-          uint32_t gv[32], uv[32];
-          load_chunk(c * 32, gv);
-          load_chunk(128 + c * 32, uv);
-          const int col0 = n0 + c * 32;
-          if (!row_ok || col0 >= g.N) continue;
-          bf16* dst = g.C + (size_t)row * g.ldc + col0;
-          if ((g.ldc & 7) == 0 && col0 + 32 <= g.N) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              Pack8 o;
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float g0 = __uint_as_float(gv[q * 8 + 2 * e]), g1 = __uint_as_float(gv[q * 8 + 2 * e + 1]);
-                const float u0 = __uint_as_float(uv[q * 8 + 2 * e]), u1 = __uint_as_float(uv[q * 8 + 2 * e + 1]);
-                o.h[e] = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
-              }
-              reinterpret_cast<uint4*>(dst)[q] = o.u;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (col0 + j < g.N) {
-                const float gg = __uint_as_float(gv[j]), uu = __uint_as_float(uv[j]);
-                dst[j] = __float2bfloat16_rn(gg / (1.f + __expf(-gg)) * uu);
-              }
-            }
-          }
-        }
+        epilogue_swiglu(load_chunk, g, ew, n0);
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {         // statistics are kept per 128 columns
@@ -513,7 +432,7 @@ int sm_count2() {
 
 template <int EPI>
 int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
-  const int smem = ST2 * STAGE2 + 1024;
+  const int smem = ST2 * STAGE2 + 1024 + 4 * kEpiStageBytes;   // stage ring, alignment slack, epilogue staging
   static bool attr_set = false;
   if (!attr_set) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
