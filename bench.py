@@ -241,7 +241,7 @@ def run_ours(args, rank, world, device):
     gemm_ms = sum(phases[k]["ms"] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) / args.steps
     gemm_flops = shape.n_layers * 2 * n * shape.params_per_layer
     # DRAM bytes of one launch from the committed ncu capture of this workload (profiles/), null elsewhere
-    traffic = 229.4e6 if wl.name == "llada1l_1024" else None
+    traffic = 229.7e6 if wl.name == "llada1l_1024" else None
     roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel<SWIGLU> (gate/up projection, 1 launch per layer)",
                 "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst",
                 "unit": "TFLOP/s", "frac": round(achieved / peaks["bf16_tflops"], 4), "traffic": traffic,

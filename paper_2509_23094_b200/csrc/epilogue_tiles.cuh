@@ -67,14 +67,15 @@ __device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const Gemm
   const int rsub = w.lane >> 2, cg = w.lane & 3;
   uint4 rc[8], rn[8];                                         // residual of this pass and of the next one
   auto load_res = [&](int p, uint4 (&r)[8]) {
-    if (EPI != EPI_RESIDUAL || !vec || p >= pairs) return;
+    if (EPI == EPI_RESIDUAL && vec && p < pairs) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+      for (int j = 0; j < 4; ++j)
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int row = w.row0 + j * 8 + rsub, col = n0 + p * 64 + h * 32 + cg * 8;
-        if (row < w.n && col + 8 <= g.N) r[j * 2 + h] = __ldcg(reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col));
-      }
+        for (int h = 0; h < 2; ++h) {
+          const int row = w.row0 + j * 8 + rsub, col = n0 + p * 64 + h * 32 + cg * 8;
+          if (row < w.n && col + 8 <= g.N) r[j * 2 + h] = __ldcg(reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col));
+        }
+    }
   };
   load_res(0, rc);
 #pragma unroll 1

@@ -110,7 +110,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
 }
 
-union Pack8 { uint4 u; __nv_bfloat162 h[4]; };
 
 struct TcParams {
   GemmArgs g;

@@ -19,7 +19,8 @@ def _bf16(shape, seed, std=1.0):
 @pytest.mark.parametrize("impl", [1, 2, 0])
 @pytest.mark.parametrize("rows,n,N,K", [(200, 200, 256, 128), (300, 131, 384, 256), (128, 128, 128, 64),
                                          (520, 517, 1000, 192), (64, 0, 256, 128), (260, 1, 128, 1024),
-                                         (256, 100, 4096, 512), (1024, 130, 2048, 256), (512, 40, 8192, 128)])
+                                         (256, 100, 4096, 512), (1024, 130, 2048, 256), (512, 40, 8192, 128),
+                                         (300, 290, 1004, 128), (600, 599, 330, 64)])
 def test_gemm_matches_fp64(impl, rows, n, N, K):
     A = _bf16((rows, K), 1); W = _bf16((N, K), 2, 0.05); bias = _bf16((N,), 3)
     n_dev = torch.tensor([n], dtype=torch.int32, device="cuda")
