@@ -70,6 +70,7 @@ typedef struct {
 #define D2C_FLAG_PORTABLE_GEMM 1        /* run the GEMMs on the mma.sync kernel instead of the tcgen05 one (cross-check) */
 #define D2C_FLAG_PORTABLE_ATTENTION 2   /* same for the attention kernels                                                */
 #define D2C_FLAG_ONE_SM_GEMM 4          /* keep the GEMMs on the one-SM tcgen05 kernel (no CTA pairs)                    */
+#define D2C_FLAG_SERIAL 8               /* enqueue every kernel of a step on the caller's stream, one after the other    */
 
 /* Weights.  The arrays of per-layer pointers are HOST arrays of n_layers DEVICE
  * pointers; they are copied at create, the device memory is borrowed for the

@@ -99,7 +99,7 @@ static const char* check_config(const d2c_config* c) {
   if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
   if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
   if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
-  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION | D2C_FLAG_ONE_SM_GEMM))) return "rollout_layers >= 0 and no unknown flag bits required";
+  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION | D2C_FLAG_ONE_SM_GEMM | D2C_FLAG_SERIAL))) return "rollout_layers >= 0 and no unknown flag bits required";
   return nullptr;
 }
 
@@ -122,6 +122,13 @@ struct d2c_ctx {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t layers_done = nullptr;
   void* early_hidden_host = nullptr;     // set by d2c_step_host for the duration of one step
+  // The head-averaged probabilities and the rollout feed only the next step's selection.  They run on a
+  // low-priority stream beside the projections, the FFN and the LM head, filling the SMs those leave idle
+  // (partial last waves); the rest of the step runs on a high-priority stream so that it wins every SM it
+  // can use.  Both are forked from and joined to the caller's stream by events inside d2c_step.
+  cudaStream_t work_stream = nullptr, side_stream = nullptr;
+  cudaEvent_t ev_in = nullptr, ev_out = nullptr, ev_fwd = nullptr, ev_abar = nullptr, ev_side = nullptr;
+  cudaStream_t run = nullptr;            // where the current step's critical path is enqueued
   char err[512];
   // optional per-phase timing: one event at every phase boundary, resolved by d2c_profile_read
   bool prof = false;
@@ -133,6 +140,16 @@ struct d2c_ctx {
   long long launch_mark = 0;
   int prof_phase = -1;
 };
+
+static void destroy_overlap(d2c_ctx* ctx) {
+  if (ctx->work_stream) cudaStreamDestroy(ctx->work_stream);
+  if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
+  for (cudaEvent_t* ev : {&ctx->ev_in, &ctx->ev_out, &ctx->ev_fwd, &ctx->ev_abar, &ctx->ev_side}) {
+    if (*ev) cudaEventDestroy(*ev);
+    *ev = nullptr;
+  }
+  ctx->work_stream = ctx->side_stream = nullptr;
+}
 
 // Marks the start of `phase` (or the end of the step with phase < 0) on the context's stream.
 static int mark(d2c_ctx* ctx, int phase) {
@@ -164,7 +181,7 @@ static int pass(d2c_ctx* ctx, int rc) {
 }
 // The step's GEMMs: tcgen05 kernel unless the context was created with D2C_FLAG_PORTABLE_GEMM.
 static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
-  if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->stream);
+  if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->run);
   // The LM head runs on few rows and is bound by the weight stream: the one-SM kernel sizes its A boxes to the
   // live rows, a pair would load a second, empty row tile.
   const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;   // weight-streaming regime
@@ -172,11 +189,17 @@ static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   {
     GemmArgs g2 = g;
     g2.sk_partials = ctx->buf.sk_partials; g2.sk_counters = ctx->buf.sk_counters; g2.sk_max_tiles = kSkMaxTiles;
-    return launch_gemm_tc2(g2, epi, ctx->stream, ctx->buf.status);
+    return launch_gemm_tc2(g2, epi, ctx->run, ctx->buf.status);
   }
   GemmArgs gs = g;
   gs.sk_partials = ctx->buf.sk_partials; gs.sk_counters = ctx->buf.sk_counters; gs.sk_max_tiles = kSkMaxTiles;
-  return launch_gemm_tc(gs, epi, ctx->stream, ctx->buf.status);
+  return launch_gemm_tc(gs, epi, ctx->run, ctx->buf.status);
+}
+// A CUDA runtime call inside the step: its error text goes where launcher errors go.
+static int cu(cudaError_t e) {
+  if (e == cudaSuccess) return D2C_OK;
+  set_global_error("d2c_step: %s", cudaGetErrorString(e));
+  return D2C_ECUDA;
 }
 #define D2C_TRY(ctx, expr) do { int rc__ = (expr); if (rc__ != D2C_OK) return pass((ctx), rc__); } while (0)
 
@@ -223,6 +246,16 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     ctx->copy_stream = nullptr; ctx->layers_done = nullptr; (void)cudaGetLastError();
   }
+  ctx->run = ctx->stream;
+  if (!(cfg->flags & D2C_FLAG_SERIAL)) {
+    int least = 0, greatest = 0;
+    bool ok = cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess && greatest < least &&
+              cudaStreamCreateWithPriority(&ctx->work_stream, cudaStreamNonBlocking, greatest) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&ctx->side_stream, cudaStreamNonBlocking, least) == cudaSuccess;
+    for (cudaEvent_t* ev : {&ctx->ev_in, &ctx->ev_out, &ctx->ev_fwd, &ctx->ev_abar, &ctx->ev_side})
+      ok = ok && cudaEventCreateWithFlags(ev, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { destroy_overlap(ctx); (void)cudaGetLastError(); }      // the step then runs on the caller's stream alone
+  }
   cudaError_t e = cudaMemsetAsync(workspace, 0, need, ctx->stream);
   if (e == cudaSuccess) {
     std::vector<uint32_t> tab(cfg->max_seq);
@@ -245,6 +278,7 @@ int d2c_destroy(d2c_ctx* ctx) {
   if (ctx->n_hint) cudaFreeHost(ctx->n_hint);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->layers_done) cudaEventDestroy(ctx->layers_done);
+  destroy_overlap(ctx);
   delete ctx;
   return D2C_OK;
 }
@@ -288,7 +322,26 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   D2C_TRY(ctx, check_step_args(ctx, a));
   const d2c_config& c = ctx->cfg;
   const Buffers& b = ctx->buf;
-  cudaStream_t st = ctx->stream;
+  // critical path on `st`, probabilities + rollout on `side` (the same stream while profiling or when serial)
+  const bool overlap = ctx->work_stream != nullptr && !ctx->prof;
+  cudaStream_t st = overlap ? ctx->work_stream : ctx->stream;
+  cudaStream_t side = overlap ? ctx->side_stream : st;
+  ctx->run = st;
+  if (overlap) {
+    D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_in, ctx->stream)));
+    D2C_TRY(ctx, cu(cudaStreamWaitEvent(st, ctx->ev_in, 0)));
+  }
+  // The probabilities pass of a layer goes to the side stream when its CTAs cannot hold up the projections
+  // that follow: in the weight-streaming regime (few rows: short CTAs, GEMMs bound by HBM) and for a single
+  // layer (it then overlaps the LM head).  Otherwise a statically scheduled GEMM whose CTAs start late behind
+  // side-stream CTAs loses more than the overlap gains (measured at 488 rows x 32 layers: +5 %).
+  const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;
+  const bool abar_aside = overlap && (c.n_layers == 1 || few_rows);
+  bool abar_pending = false, rollout_done = false;
+  // Eq. 6-9 for the next step's stage 2: enqueued right after the last probabilities pass it needs
+  RolloutArgs r{};
+  r.abar = b.abar; r.layer_stride = (size_t)c.max_batch * c.max_seq * c.max_seq; r.n_layers = rollout_depth(c); r.sel_idx = b.sel_idx;
+  r.row_off = b.row_off; r.batch = a->batch; r.seq_len = a->seq_len; r.c = b.c; r.u0 = b.u0; r.u1 = b.u1; r.partial = b.partial; r.n_split = kRolloutSplit;
   const int B = a->batch, L = a->seq_len, R = B * L, d = c.d_model;
   const int hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
   const int qkv_out = (hq + 2 * hkv) * dh;
@@ -322,6 +375,10 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
       D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
     }
     D2C_TRY(ctx, mark(ctx, PH_QKV));
+    if (abar_pending) {                                  // the previous layer's probabilities still read Q and the LSE
+      D2C_TRY(ctx, cu(cudaStreamWaitEvent(st, ctx->ev_abar, 0)));
+      abar_pending = false;
+    }
     GemmArgs g{};
     g.A = b.xn; g.lda = d; g.W = ctx->wqkv[l]; g.bias = ctx->bqkv[l]; g.C = b.qkv; g.ldc = qkv_out;
     g.n_rows = n_rows; g.max_rows = R; g.N = qkv_out; g.K = d;
@@ -348,7 +405,25 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     if (at.abar) {
       D2C_TRY(ctx, mark(ctx, PH_ABAR));
       at.which = 2;
-      D2C_TRY(ctx, launch_attention(at, st));
+      if (abar_aside) {
+        D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_fwd, st)));
+        D2C_TRY(ctx, cu(cudaStreamWaitEvent(side, ctx->ev_fwd, 0)));
+      }
+      D2C_TRY(ctx, launch_attention(at, abar_aside ? side : st));
+      if (abar_aside) {
+        D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_abar, side)));
+        abar_pending = true;
+      }
+      if (l == depth - 1) {
+        D2C_TRY(ctx, mark(ctx, PH_ROLLOUT));
+        if (overlap && !abar_aside) {                    // the side stream has followed nothing of this step yet
+          D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_fwd, st)));
+          D2C_TRY(ctx, cu(cudaStreamWaitEvent(side, ctx->ev_fwd, 0)));
+        }
+        D2C_TRY(ctx, launch_rollout(r, side));
+        if (overlap) D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_side, side)));
+        rollout_done = true;
+      }
     }
     D2C_TRY(ctx, mark(ctx, PH_O));
     GemmArgs go{};
@@ -383,12 +458,8 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   gl.logits = out ? out->logits : nullptr;
   D2C_TRY(ctx, gemm(ctx, gl, EPI_LMSTATS));
   D2C_TRY(ctx, launch_lm_reduce(b.st_max, b.st_sum, b.st_arg, gl.n_tiles, n_lm, R, b.lm_rows, b.sel_idx, b.row_seq, L, b.conf, b.pred, st));
-  // Eq. 6-9 for the next step's stage 2
-  D2C_TRY(ctx, mark(ctx, PH_ROLLOUT));
-  RolloutArgs r{};
-  r.abar = b.abar; r.layer_stride = (size_t)c.max_batch * c.max_seq * c.max_seq; r.n_layers = depth; r.sel_idx = b.sel_idx;
-  r.row_off = b.row_off; r.batch = B; r.seq_len = L; r.c = b.c; r.u0 = b.u0; r.u1 = b.u1; r.partial = b.partial; r.n_split = kRolloutSplit;
-  D2C_TRY(ctx, launch_rollout(r, st));
+  if (!rollout_done) return fail(ctx, D2C_EINVAL, "d2c_step: no layer produced attention probabilities");
+  if (overlap) D2C_TRY(ctx, cu(cudaStreamWaitEvent(st, ctx->ev_side, 0)));
 
   D2C_TRY(ctx, mark(ctx, PH_OUT));
   if (out && out->sel_idx) {
@@ -404,6 +475,11 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
   }
   D2C_TRY(ctx, mark(ctx, -1));
+  if (overlap) {
+    D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_out, st)));
+    D2C_TRY(ctx, cu(cudaStreamWaitEvent(ctx->stream, ctx->ev_out, 0)));
+  }
+  ctx->run = ctx->stream;
   return D2C_OK;
 }
 

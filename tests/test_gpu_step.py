@@ -237,6 +237,25 @@ def test_kernel_variants_agree():
             assert row_rel_err(g["hidden"][b], ref["hidden"][b].astype(np.float64)) <= ROW_TOL
 
 
+def test_overlapped_and_serial_steps_are_identical():
+    """The probabilities / rollout side stream changes when kernels run, not what they compute."""
+    wl = inputs.Workload("hd128_overlap", inputs.TOY_HD128, 2, 300, 150, 60, "random", 8, 0.6, seed=11)
+    got = []
+    for flags in (0, 8):                                              # default (two streams); D2C_FLAG_SERIAL
+        pair = Pair(wl, flags=flags)
+        pair.gpu_step(10 ** 6, 1.0)
+        steps = [pair.gpu_step(wl.k, wl.p) for _ in range(3)]         # each step selects from the previous step's rollout
+        B, L = wl.batch, wl.seq_len
+        got.append((steps, pair.ctx.view("c", B, L).clone(), pair.ctx.view("conf", B, L).clone(),
+                    pair.ctx.view("kcache").clone()))
+    (sa, ca, fa, ka), (sb, cb, fb, kb) = got
+    for ga, gb in zip(sa, sb):
+        for b in range(wl.batch):
+            np.testing.assert_array_equal(ga["sel"][b], gb["sel"][b])
+            np.testing.assert_array_equal(ga["hidden"][b], gb["hidden"][b])
+    assert torch.equal(ca, cb) and torch.equal(fa, fb) and torch.equal(ka, kb)
+
+
 def test_semi_autoregressive_block_restricts_stage1():
     from oracle import selection as osel
     wl = inputs.Workload("semiar", inputs.TOY_HD128, 2, 192, 64, 128, "all", 6, 0.4, seed=5)
