@@ -25,9 +25,13 @@
  *     comment says "host".  The library allocates no device memory: weights, the
  *     workspace and all outputs belong to the caller.
  *   - bf16 matrices are row-major [out_features][in_features].
- *   - All work is enqueued on the stream given to d2c_create; calls return
- *     without synchronising unless stated.  One context per stream; a context is
- *     not re-entrant.
+ *   - All work is ordered on the stream given to d2c_create; calls return
+ *     without synchronising unless stated.  d2c_step may run part of a step on
+ *     two streams of its own (created by d2c_create, forked from and joined to
+ *     the caller's stream by events inside the call), so work enqueued on the
+ *     caller's stream after the call still sees the whole step; D2C_FLAG_SERIAL
+ *     keeps every kernel on the caller's stream (needed for stream capture).
+ *     One context per stream; a context is not re-entrant.
  *   - Return value: D2C_OK or a negative D2C_E* code; d2c_last_error() gives the
  *     text.  Nothing throws, aborts or traps.  Faults detected on the device
  *     (a bounded wait that ran out) are written to a status word that
