@@ -154,6 +154,11 @@ def run_ours(args, rank, world, device):
     ctx.step(h0, mask_dev, 10 ** 6, 1.0)
     ctx.sync_status()
     snap = {n: ctx.view(n, B, L).clone() for n in ("conf", "pred", "c")}
+    if args.scores == "zipf":
+        # paper-like peaked stage-2 scores instead of the nearly flat ones random weights give: seeded Zipf(1.0)
+        # over the positions of every sequence; top-p then keeps few rows for the same p
+        for b in range(B):
+            snap["c"][b] = inputs.make_scores(L, seed=wl.seed + 1000 + b, kind="zipf").to(device)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)       # > L2 (126 MB)
     hid = torch.zeros(B * L, d, dtype=torch.bfloat16, device=device)
 
@@ -264,7 +269,7 @@ def run_ours(args, rank, world, device):
         "config": {"workload": wl.name, "shape": shape.name, "batch": B, "seq_len": L, "k": wl.k, "p": wl.p,
                    "selected_rows": n_b, "lm_rows": n_m, "l2": "flushed between steps; weights (%.2f GB) exceed L2" %
                    ((2 * shape.n_layers * shape.params_per_layer + 2 * d * shape.vocab) / 1e9),
-                   "replicas": world},
+                   "replicas": world, "scores": args.scores},
         "clocks": clocks,
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": round(e2e_s / e2e_steps * 1e3, 4)},
@@ -400,6 +405,8 @@ def main():
     ap.add_argument("--decode", action="store_true", help="also run the workload's whole decoding loop")
     ap.add_argument("--p", type=float, default=None, help="override the workload's top-p threshold (e.g. the paper's default 0.1)")
     ap.add_argument("--k", type=int, default=None, help="override the workload's k")
+    ap.add_argument("--scores", default="rollout", choices=["rollout", "zipf"],
+                    help="stage-2 scores before each timed step: the prefill's rollout (default) or a seeded Zipf(1.0)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
