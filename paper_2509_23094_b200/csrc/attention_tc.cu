@@ -117,6 +117,11 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
 constexpr uint32_t kIdescKK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescKMn = kIdescKK | (1u << 16);
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
@@ -273,12 +278,21 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         for (int c = 0; c < 4; ++c) tmem_ld32(ts + c * 32, sv[c]);
         tmem_ld_wait();
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (full) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 4; ++c) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float f = __uint_as_float(sv[c][i]);
-            if (full || key0 + c * 32 + i < L) mx4[i & 3] = fmaxf(mx4[i & 3], f);
+            for (int i = 0; i < 32; i += 2)                             // three-input maximum: two scores per instruction
+              mx4[(i >> 1) & 3] = fmax3(mx4[(i >> 1) & 3], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float f = __uint_as_float(sv[c][i]);
+              if (key0 + c * 32 + i < L) mx4[i & 3] = fmaxf(mx4[i & 3], f);
+            }
           }
         }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
