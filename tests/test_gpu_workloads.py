@@ -152,6 +152,30 @@ def test_llada_single_layer_1024():
     assert 700 < len(S[0]) < 950                                         # flat scores: about 32 + 0.9 * 896 rows
 
 
+def test_llada_single_layer_1024_few_rows():
+    """The paper's default threshold p = 0.1: about a hundred selected rows, the weight-streaming regime.  The
+    library switches kernels (one-SM GEMM with narrow tiles and split-K, probabilities pass on the side stream)
+    on the row count of an earlier step, so the checked step is the second one with that count."""
+    wl = inputs.WORKLOADS["llada1l_1024"]
+    r = Runner(wl)
+    B, L = wl.batch, wl.seq_len
+    ro, S = r.step(10 ** 6, 1.0)
+    snap = {n: r.ctx.view(n, B, L).clone() for n in ("conf", "pred", "c")}
+    for _ in range(2):
+        for n, t in snap.items():
+            r.ctx.view(n, B, L).copy_(t)
+        kc0 = r.ctx.view("kcache").clone(); vc0 = r.ctx.view("vcache").clone()
+        ro, S = r.step(wl.k, 0.1)
+        torch.cuda.synchronize()
+    assert 64 < len(S[0]) <= 128                                         # flat scores: about 32 + 0.1 * 896 rows
+    r.check_layers(ro, S, [0], seqs=[0])
+    r.check_lm_head()
+    r.check_rollout(ro, S, [0])
+    kc1 = r.ctx.view("kcache"); vc1 = r.ctx.view("vcache")
+    keep = torch.ones(L, dtype=torch.bool, device="cuda"); keep[torch.from_numpy(S[0]).cuda()] = False
+    assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
+
+
 def test_llada_32_layers_768_with_a_committed_token():
     r, ro, S, _ = _run("llada_decode", [0, 1, 16, 31], [0, 31], [0])
     # decode-loop shape: commit the most confident masked row, force it into the next step
