@@ -12,9 +12,8 @@
 //
 // Warp roles in both: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2.. softmax/epilogue.
 // No cluster, no multicast.  Every mbarrier wait is bounded (see gemm_tc.cu for the protocol).
-#include <cuda.h>
-
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace d2c {
 namespace {
@@ -22,91 +21,22 @@ namespace {
 constexpr int AQ = 128, AKEYS = 128, ADH = 128;
 constexpr int HALF_BYTES = 128 * 64 * 2;          // one 128-row x 64-column swizzled box: 16 KB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;        // 128 x 128 bf16
-constexpr long long kWaitCycles = 4000000000LL;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
 __device__ int g_attn_status[4];
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile("{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
-               : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-  return done;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = site;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
+// D (TMEM) (+)= A (TMEM) x B (shared memory): the probabilities stay in TMEM
 __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
                ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                 "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                 "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                 "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-               : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
                  "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// K-major bf16 tile of 128-byte swizzled rows (8-row groups 1024 bytes apart).
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
-         ((uint64_t)2 << 61);
-}
 // MN-major bf16 operand: 64 contiguous N elements per 128-byte row, 8 K-rows per 1024-byte group
 // (stride offset), the next 64 N elements 16 KB further (leading offset).
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
@@ -230,7 +160,7 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 #pragma unroll
         for (int i = 0; i < ADH / 16; ++i) {
           const uint32_t off = (i >> 2) * HALF_BYTES;
-          umma_ss(tm + q * 256, desc_kmajor(sQ(q) + off) + 2 * (i & 3), desc_kmajor(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
+          umma_ss(tm + q * 256, smem_desc_sw128(sQ(q) + off) + 2 * (i & 3), smem_desc_sw128(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
         }
         umma_commit(B(7 + q));
       };
@@ -458,7 +388,7 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
         for (int i = 0; i < ADH / 16; ++i) {
           const uint32_t off = (i >> 2) * HALF_BYTES;
-          umma_ss(tm + sb * 128, desc_kmajor(sQ(s) + off) + 2 * (i & 3), desc_kmajor(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
+          umma_ss(tm + sb * 128, smem_desc_sw128(sQ(s) + off) + 2 * (i & 3), smem_desc_sw128(sK(ks) + off) + 2 * (i & 3), kIdescKK, i != 0);
         }
         umma_commit(QE(s));                                         // Q stage free
         if ((h + 1) % group == 0 || h + 1 == nh) umma_commit(KE(ks));        // last head of the group: K stage free
@@ -533,34 +463,6 @@ abar_sum_kernel(const float* __restrict__ part, size_t group_stride, int groups,
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-// [rows][cols] bf16, leading dimension ld, box 128 rows x 64 columns, 128-byte swizzle, zero fill.
-int make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) { set_global_error("cuTensorMapEncodeTiled is not available from this driver"); return D2C_ECUDA; }
-  const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {ld * 2};
-  const cuuint32_t box[2] = {64, 128};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) { set_global_error("cuTensorMapEncodeTiled failed with code %d", (int)r); return D2C_ECUDA; }
-  return D2C_OK;
-}
 }  // namespace
 
 // True if the tcgen05 kernels can take this problem (otherwise the caller uses the mma.sync ones).
@@ -580,9 +482,9 @@ int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   }
   CUtensorMap tmQ, tmK, tmV;
   const uint64_t kv_cols = (uint64_t)a.hkv * a.dh, kv_rows = (uint64_t)a.batch * a.cache_seq;
-  int rc = make_map(&tmQ, a.q, (uint64_t)a.q_rows, (uint64_t)a.hq * a.dh, (uint64_t)a.ldq);
-  if (rc == D2C_OK) rc = make_map(&tmK, a.kc, kv_rows, kv_cols, kv_cols);
-  if (rc == D2C_OK) rc = make_map(&tmV, a.vc, kv_rows, kv_cols, kv_cols);
+  int rc = make_bf16_map(&tmQ, a.q, (uint64_t)a.q_rows, (uint64_t)a.hq * a.dh, (uint64_t)a.ldq, 128);
+  if (rc == D2C_OK) rc = make_bf16_map(&tmK, a.kc, kv_rows, kv_cols, kv_cols, 128);
+  if (rc == D2C_OK) rc = make_bf16_map(&tmV, a.vc, kv_rows, kv_cols, kv_cols, 128);
   if (rc != D2C_OK) return rc;
   int sms = 148, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 148;
