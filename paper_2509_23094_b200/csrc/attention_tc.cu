@@ -165,7 +165,40 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         umma_commit(B(7 + q));
       };
       bool ok = mbar_wait(B(0), 0, abortp, status, 12) && mbar_wait(B(1), 0, abortp, status, 13);
-      if (ok) {
+      if (nq == 1) {
+        // One live query tile: the second tile's TMEM columns are free, so the scores of key tile j + 1 are
+        // computed there while the softmax warps work on tile j (S/P buffer = j & 1, O stays in the first half).
+        auto issue_s1 = [&](int j) {
+          const int s = j & 1;
+#pragma unroll
+          for (int i = 0; i < ADH / 16; ++i) {
+            const uint32_t off = (i >> 2) * HALF_BYTES;
+            umma_ss(tm + s * 256, smem_desc_sw128(sQ(0) + off) + 2 * (i & 3), smem_desc_sw128(sK(s) + off) + 2 * (i & 3), kIdescKK, i != 0);
+          }
+          umma_commit(B(7 + s));
+        };
+        if (ok) {
+          tc_fence_after();
+          issue_s1(0);
+        }
+        for (int j = 0; j < T && ok; ++j) {
+          const int s = j & 1, u = j >> 1;
+          if (j + 1 < T) {
+            if (!mbar_wait(B(1 + ((j + 1) & 1)), ((j + 1) >> 1) & 1, abortp, status, 16)) { ok = false; break; }
+            tc_fence_after();
+            issue_s1(j + 1);                                        // its buffer held P_{j-1}, consumed by the product issued before
+          }
+          if (!mbar_wait(B(9 + s), u & 1, abortp, status, 14)) { ok = false; break; }
+          if (!mbar_wait(B(3 + s), u & 1, abortp, status, 15)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int i = 0; i < AKEYS / 16; ++i)
+            umma_ts(tm + 128, tm + s * 256 + 8 * i, desc_mnmajor(sV(s) + i * 2048), kIdescKMn, (j | i) != 0);
+          umma_commit(B(11));
+          umma_commit(B(5 + s));
+        }
+        ok = false;                                                 // done: skip the two-tile schedule below
+      } else if (ok) {
         tc_fence_after();
         for (int q = 0; q < nq; ++q) issue_s(q, 0);
       }
@@ -194,12 +227,15 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (q < nq) {
       const int quarter = warp & 3, lrow = q * AQ + quarter * 32 + lane;
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-      const uint32_t ts = tm + q * 256 + lane_base, to = ts + 128;
+      const bool dbuf = nq == 1;                                    // one query tile: S/P alternate between the TMEM halves
+      const uint32_t to = tm + q * 256 + 128 + lane_base;
       const float sc = kLog2e * rsqrtf((float)ADH);
       float m_used = -INFINITY, l = 0.f;
       bool ok = true;
       for (int j = 0; j < T && ok; ++j) {
-        if (!mbar_wait(B(7 + q), j & 1, abortp, status, 18)) { ok = false; break; }
+        const int sp = dbuf ? (j & 1) : q;                          // S/P buffer of this tile
+        const uint32_t ts = tm + sp * 256 + lane_base;
+        if (!mbar_wait(B(7 + sp), (dbuf ? (j >> 1) : j) & 1, abortp, status, 18)) { ok = false; break; }
         tc_fence_after();
         const int key0 = j * AKEYS;
         const bool full = key0 + AKEYS <= L;
@@ -269,7 +305,7 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(B(9 + q));
+        if (lane == 0) mbar_arrive(B(9 + sp));
       }
       if (ok) ok = mbar_wait(B(11 + q), (T - 1) & 1, abortp, status, 19);
       tc_fence_after();
