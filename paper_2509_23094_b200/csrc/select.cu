@@ -16,10 +16,18 @@ namespace d2c {
 static constexpr int kSelThreads = 1024;
 enum : uint8_t { F_SEL = 1, F_MSTAR = 2 };
 
+// Descending bitonic sort of n 64-bit words in shared memory by the whole block.  Pair p of a stage exchanges
+// elements lo = 2p - (p & (stride - 1)) and lo + stride; for stride <= 32 the pairs of one warp touch only that
+// warp's 64 elements, so only the stages that reach further need the block to synchronise.  (Keeping the words in
+// registers and exchanging by warp shuffles was no faster: with 32 warps on one SM the stages are bound by
+// instruction issue, not by the shared-memory round trip.)
 __device__ __forceinline__ void bitonic_sort_desc(uint64_t* buf, int n) {
+  bool wide_before = true;                                  // the caller's writes count as a block-wide stage
   for (int size = 2; size <= n; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      __syncthreads();
+      const bool wide = stride >= 64;
+      if (wide || wide_before) __syncthreads(); else __syncwarp();
+      wide_before = wide;
       for (int t = threadIdx.x; t < (n >> 1); t += blockDim.x) {
         const int lo = 2 * t - (t & (stride - 1));
         const int hi = lo + stride;

@@ -51,7 +51,7 @@ def test_random_cases(seed):
               kind=["uniform", "zipf", "flat"][seed % 3], ties=[0, 16, 3][seed % 3], mode=seed % 2)
 
 
-@pytest.mark.parametrize("L", [1, 31, 32, 33, 127, 128, 129, 1024, 1025, 4096])
+@pytest.mark.parametrize("L", [1, 31, 32, 33, 127, 128, 129, 600, 1024, 1025, 2048, 4096, 5000, 8192])
 def test_sizes_around_tile_boundaries(L):
     _run_case(2, L, 0.3, 32, 0.9, L, kind="flat")
     _run_case(1, L, 0.5, 8, 0.1, L + 1, kind="zipf", use_key=True)
