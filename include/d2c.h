@@ -30,7 +30,9 @@
  *     two streams of its own (created by d2c_create, forked from and joined to
  *     the caller's stream by events inside the call), so work enqueued on the
  *     caller's stream after the call still sees the whole step; D2C_FLAG_SERIAL
- *     keeps every kernel on the caller's stream (needed for stream capture).
+ *     keeps every kernel on the caller's stream.  Either way a step can be captured
+ *     into a CUDA graph from the caller's stream and replayed (the choice between
+ *     kernel variants that follows an earlier step's row count is then frozen).
  *     One context per stream; a context is not re-entrant.
  *   - Return value: D2C_OK or a negative D2C_E* code; d2c_last_error() gives the
  *     text.  Nothing throws, aborts or traps.  Faults detected on the device

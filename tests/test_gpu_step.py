@@ -256,6 +256,43 @@ def test_overlapped_and_serial_steps_are_identical():
     assert torch.equal(ca, cb) and torch.equal(fa, fb) and torch.equal(ka, kb)
 
 
+@pytest.mark.parametrize("flags", [0, 8])
+def test_step_replayed_from_a_cuda_graph(flags):
+    """d2c_step captured into a CUDA graph (with and without the internal streams) replays to the same bits."""
+    wl = inputs.Workload("hd128_graph", inputs.TOY_HD128, 2, 300, 150, 60, "random", 8, 0.6, seed=12)
+    B, L, d = wl.batch, wl.seq_len, wl.shape.d_model
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        pair = Pair(wl, flags=flags)
+        pair.gpu_step(10 ** 6, 1.0)
+        snap = {n: pair.ctx.view(n, B, L).clone() for n in ("conf", "pred", "c")}
+        kc = pair.ctx.view("kcache").clone(); vc = pair.ctx.view("vcache").clone()
+
+        def restore():
+            for n, t in snap.items():
+                pair.ctx.view(n, B, L).copy_(t)
+            pair.ctx.view("kcache").copy_(kc); pair.ctx.view("vcache").copy_(vc)
+
+        h0, mask = pair.h0.cuda(), pair.mask.cuda()
+        hid = torch.zeros(B * L, d, dtype=torch.bfloat16, device="cuda")
+        restore()
+        pair.ctx.step(h0, mask, wl.k, wl.p, hidden_out=hid)           # eager: also the first launch of every kernel
+        pair.ctx.sync_status()
+        want = (hid.clone(), pair.ctx.view("c", B, L).clone(), pair.ctx.view("conf", B, L).clone(),
+                pair.ctx.view("kcache").clone())
+        restore(); hid.zero_()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            pair.ctx.step(h0, mask, wl.k, wl.p, hidden_out=hid)
+        for _ in range(2):
+            restore(); hid.zero_()
+            graph.replay()
+            pair.ctx.sync_status()
+            got = (hid, pair.ctx.view("c", B, L), pair.ctx.view("conf", B, L), pair.ctx.view("kcache"))
+            assert all(torch.equal(a, b) for a, b in zip(got, want))
+
+
 def test_semi_autoregressive_block_restricts_stage1():
     from oracle import selection as osel
     wl = inputs.Workload("semiar", inputs.TOY_HD128, 2, 192, 64, 128, "all", 6, 0.4, seed=5)
