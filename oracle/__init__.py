@@ -13,7 +13,9 @@ Pin status (see tests/test_oracle_*.py):
   model.* (select-all)                an independently written torch fp64 textbook forward
   model.lm_head_conf                  softmax identities, zero-weight closed form
   step.oracle_step                    select-all == no-cache forward; select-none == identity;
-                                      single-layer exactness
-  step.oracle_step with a strict subset of rows on N >= 2 layers: parity unpinned
-  beyond the pieces above (the paper prints no worked example of the approximation).
+                                      single-layer exactness; a strict subset of rows on two and
+                                      three layers with a stale cache == an independently written
+                                      torch fp64 subset step (index assignment into the cache, library
+                                      attention over all keys); rollout_layers = n == Eq. 6-9 over the
+                                      first n layers of the same step (and differs from the last n)
 """
