@@ -11,6 +11,52 @@ from paper_2509_23094_b200 import binding, inputs
 # max |gpu - oracle| over a row, relative to the oracle row's L2 norm (bf16 storage, fp32 accumulation)
 ROW_TOL = 2e-2
 
+# Worst error seen per tensor in this process (printed in the terminal summary), and regression bounds:
+# about four times the worst error the committed kernels showed on a B200 over the whole GPU suite.  A
+# row-norm tolerance of 2e-2 at 4096 columns admits one element that is off by more than a row RMS; the
+# regression bound is what catches a kernel that starts to drift or gets single elements wrong.
+OBSERVED = {}
+# (observed over the suite: K 2.2e-3, V 2.4e-3, hidden 2.0e-3, abar 3.2e-3, logits 8.6e-4, c 5.1e-4)
+REGRESSION = {"K": 9e-3, "V": 1e-2, "hidden": 8e-3, "abar": 1.3e-2, "logits": 3.5e-3, "c": 2e-3}
+
+
+def observe(name: str, err: float) -> float:
+    OBSERVED[name] = max(OBSERVED.get(name, 0.0), float(err))
+    return float(err)
+
+
+def check_rows(name: str, got, want, what="") -> float:
+    """Row-norm-relative error of one tensor kind: recorded, held to the stated tolerance and to its regression bound."""
+    err = observe(name, row_rel_err(np.asarray(got), np.asarray(want)))
+    assert err <= ROW_TOL, (name, what, err)
+    assert err <= REGRESSION[name], (name, what, err, "regression bound")
+    return err
+
+
+def check_scores(got, want, what="") -> float:
+    """Rollout scores c (Eq. 9): element-wise relative error."""
+    got = np.asarray(got, dtype=np.float64); want = np.asarray(want, dtype=np.float64)
+    err = observe("c", float(np.max(np.abs(got - want) / np.maximum(np.abs(want), 1e-4)))) if want.size else 0.0
+    assert err <= 2e-2 and err <= REGRESSION["c"], ("c", what, err)
+    return err
+
+
+def check_lm_rows(gpu_logits, oracle_logits, pred, conf, oracle_conf, what="") -> float:
+    """Eq. 1 on a set of rows.  The GPU's token must be the exact arg-max of the GPU's own logits (lowest id
+    among equals); its logits must match the oracle's row within the tolerance; and in the oracle's logits
+    the GPU's token may trail the oracle's best by no more than four times the observed logit error."""
+    gpu_logits = np.asarray(gpu_logits, dtype=np.float64); oracle_logits = np.asarray(oracle_logits, dtype=np.float64)
+    if oracle_logits.shape[0] == 0:
+        return 0.0
+    pred = np.asarray(pred, dtype=np.int64)
+    np.testing.assert_array_equal(pred, np.argmax(gpu_logits, axis=1), err_msg=f"{what}: pred is not the arg-max of the kernel's own logits")
+    err = check_rows("logits", gpu_logits, oracle_logits, what)
+    abs_err = np.max(np.abs(gpu_logits - oracle_logits), axis=1)
+    r = np.arange(len(pred))
+    assert np.all(oracle_logits[r, pred] >= oracle_logits.max(axis=1) - 4.0 * abs_err), (what, "predicted token is not a near-maximum of the oracle's logits")
+    np.testing.assert_allclose(conf, oracle_conf, rtol=0.1, atol=1e-7)
+    return err
+
 
 def row_rel_err(got: np.ndarray, want: np.ndarray) -> float:
     """max over rows of max|got-want| / ||want row||_2 (rows = all but the last axis flattened)."""

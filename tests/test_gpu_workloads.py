@@ -15,7 +15,7 @@ from oracle import model as omodel
 from oracle import rollout as orollout
 from oracle import selection as osel
 from paper_2509_23094_b200 import binding, inputs
-from gpu_util import ROW_TOL, row_rel_err
+from gpu_util import ROW_TOL, check_lm_rows, check_rows, check_scores, row_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -37,6 +37,8 @@ class Runner:
         B, L, d = wl.batch, wl.seq_len, wl.shape.d_model
         self.hid = torch.zeros(B * L, d, dtype=torch.bfloat16, device=dev)
         self.layer_in = torch.zeros(wl.shape.n_layers, B * L, d, dtype=torch.bfloat16, device=dev)
+        # debug output of Eq. 1: fp32 logits of every row that went through the LM head, in row order
+        self.logits = torch.zeros(int(self.mask.sum()), wl.shape.vocab, dtype=torch.float32, device=dev)
 
     def step(self, k, p, forced=None):
         wl = self.wl
@@ -48,7 +50,8 @@ class Runner:
             flat = [x for fb in forced for x in fb]
             f = torch.tensor(flat if flat else [0], dtype=torch.int32, device="cuda")
             fo = torch.tensor(np.cumsum([0] + [len(fb) for fb in forced]), dtype=torch.int32, device="cuda")
-        self.ctx.step(self.h0, self.mask.cuda(), k, p, forced=f, forced_off=fo, hidden_out=self.hid, layer_in=self.layer_in)
+        self.ctx.step(self.h0, self.mask.cuda(), k, p, forced=f, forced_off=fo, hidden_out=self.hid, layer_in=self.layer_in,
+                      logits=self.logits)
         self.ctx.sync_status()
         ro = self.ctx.view("row_off", B, L).cpu().numpy()
         sel = self.ctx.view("sel_idx").cpu().numpy()
@@ -82,11 +85,10 @@ class Runner:
                 x_out, abar = omodel.layer_on_rows(x_in, pos, Kc, Vc, w, shape.n_q_heads, shape.n_kv_heads,
                                                    shape.head_dim, shape.rope_base, shape.rms_eps)
                 kv = shape.n_kv_heads * shape.head_dim
-                errs = [row_rel_err(Kg.reshape(-1, kv), Kc[pos].reshape(-1, kv)),
-                        row_rel_err(Vg.reshape(-1, kv), Vc[pos].reshape(-1, kv)),
-                        row_rel_err(_f64(x_next[rows]), x_out),
-                        row_rel_err(self.ctx.abar(l, ro[B], L)[rows].cpu().double().numpy(), abar)]
-                assert max(errs) <= ROW_TOL, (l, b, errs)
+                errs = [check_rows("K", Kg.reshape(-1, kv), Kc[pos].reshape(-1, kv), (l, b)),
+                        check_rows("V", Vg.reshape(-1, kv), Vc[pos].reshape(-1, kv), (l, b)),
+                        check_rows("hidden", _f64(x_next[rows]), x_out, (l, b)),
+                        check_rows("abar", self.ctx.abar(l, ro[B], L)[rows].cpu().double().numpy(), abar, (l, b))]
                 worst = max(worst, max(errs))
         return worst
 
@@ -108,9 +110,10 @@ class Runner:
                                                      shape.rms_eps)
         conf_g = self.ctx.view("conf", B, L).cpu().numpy()[seq, pos]
         pred_g = self.ctx.view("pred", B, L).cpu().numpy()[seq, pos]
-        np.testing.assert_allclose(conf_g, conf_w, rtol=0.1)
-        tol = ROW_TOL * np.linalg.norm(logits, axis=1)
-        assert np.all(logits[np.arange(len(rows)), pred_g] >= logits.max(axis=1) - 2 * tol)
+        # row j of the logits output belongs to lm_rows[j]; at full vocabulary width the predicted token is held
+        # to the exact arg-max of the kernel's own logits and to a near-maximum of the oracle's
+        gpu_logits = self.logits[torch.from_numpy(pick).cuda()].cpu().numpy()
+        check_lm_rows(gpu_logits, logits, pred_g, conf_g, conf_w, "full vocabulary")
         assert np.all(self.mask.numpy()[seq, pos] == 1)                  # Eq. 1 runs on masked rows only
 
     def check_rollout(self, ro, S, seqs):
@@ -122,6 +125,7 @@ class Runner:
                 continue
             abar = [self.ctx.abar(l, ro[B], L)[ro[b]: ro[b + 1]].cpu().double().numpy() for l in range(shape.n_layers)]
             want = orollout.chain(abar, S[b], L)
+            check_scores(c[b], want, b)
             np.testing.assert_allclose(c[b], want, rtol=2e-3, atol=1e-4)
             assert abs(c[b].sum() - L) < 1e-3 * L
 
