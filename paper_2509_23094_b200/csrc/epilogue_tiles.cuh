@@ -126,18 +126,19 @@ __device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const Gemm
   }
 }
 
-// C[row][n0 .. n0 + 128) = silu(gate) * up, gate in accumulator columns [0, 128) and up in [128, 256).
+// C[row][n0 .. n0 + oc) = silu(gate) * up, gate in accumulator columns [0, oc) and up in [oc, 2 oc); oc is a
+// multiple of 32.
 template <typename LoadChunk>
-__device__ __forceinline__ void epilogue_swiglu(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0) {
+__device__ __forceinline__ void epilogue_swiglu(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int oc) {
   const bool vec = (g.ldc & 7) == 0;
   const int rsub = w.lane >> 2, cg = w.lane & 3;
 #pragma unroll 1
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < (oc >> 5); ++c) {
     {
       uint32_t v[32];
       load_chunk(c * 32, v);
       epi_stage_put(w, 0, v);
-      load_chunk(128 + c * 32, v);
+      load_chunk(oc + c * 32, v);
       epi_stage_put(w, 1, v);
     }
     __syncwarp();

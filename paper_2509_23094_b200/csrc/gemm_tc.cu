@@ -38,7 +38,9 @@ struct TcParams {
   int* status;
 };
 
-constexpr int ST = 4;                            // stages at full tile width: 4 x (16 KB of A + 32 KB of B)
+constexpr int ST = 4;                            // ring size: 4 x (16 KB of A + 32 KB of B) = 192 KB
+constexpr int KSUB = 2;                          // 64-wide k-blocks per pipeline stage (see gemm_tc2.cu on why two)
+constexpr int kSkMaxParts = 8;                   // split-K parts per tile at most
 constexpr int ST_MAX = 12;                       // narrow tiles use smaller stages and more of them
 constexpr int ACC_COLS = 256;                    // TMEM columns of one accumulator; two are allocated
 constexpr int B_BYTES = ACC_COLS * TK * 2;
@@ -92,34 +94,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n = max(*g.n_rows, 0);
   const int MT = (n + TM - 1) / TM;
-  // Accumulator width of this launch: 256 columns, narrowed to 128 or 64 while that still leaves SMs
-  // without a tile (few live rows and a small N), so that more SMs stream the weights.
+  const int KT = g.K / TK, G = gridDim.x;
+  const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
+  // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
+  // idle SM is lost bandwidth): each tile's K range is cut into S equal parts of at least four k-blocks,
+  // handled by different CTAs.  Parts park their fp32 accumulators in scratch; the part that arrives last
+  // adds them in part order (no waiting, deterministic) and runs the epilogue.
+  auto split_of = [&](int tiles) {
+    if (!sk_ok || tiles <= 0 || tiles >= G) return 1;
+    const int s = max(1, min(min(G / tiles, KT / 4), kSkMaxParts));
+    return tiles * s <= g.sk_max_tiles ? s : 1;
+  };
+  // Accumulator width of this launch.  One thread issues every MMA and pays a fixed issue latency per k-block
+  // whatever the tile's width, so a narrow tile moves fewer weight bytes per unit of that latency: the tile
+  // stays 256 columns wide and idle SMs are filled by splitting K.  Only when K is too short to split (or the
+  // epilogue has no split form) is the tile narrowed to 128 or 64 columns.  The LM head covers several waves of
+  // tiles and is bound by HBM: 128-column tiles make its last, partial wave shorter.
   int bn = ACC_COLS;
   const int bn_min = (EPI == EPI_SWIGLU) ? 256 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? max(64, g.q_dh) : 64));
-  while (bn > bn_min && 2 * MT * ((g.N + bn - 1) / bn) <= (int)gridDim.x) bn >>= 1;
+  if (EPI == EPI_LMSTATS) {
+    if (MT * ((g.N + 255) / 256) > G) bn = 128;
+  }
+  while (bn > bn_min) {
+    const int t = MT * ((g.N + bn - 1) / bn);
+    if (2 * t * split_of(t) <= G) bn >>= 1; else break;
+  }
   const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
   const int total = MT * NT;                                 // 0 when no row is live: every role loop is empty
-  const int KT = g.K / TK, G = gridDim.x;
-  // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
-  // idle SM is lost bandwidth): each tile's K range is cut into S equal parts handled by different CTAs.
-  // Parts park their fp32 accumulators in scratch; the part that arrives last adds them in part order
-  // (no waiting, deterministic) and runs the epilogue.
-  int S = 1;
-  if (g.sk_partials != nullptr && g.sk_counters != nullptr && total > 0 && total < G && total <= g.sk_max_tiles)
-    S = max(1, min(min(G / total, KT / 8), 4));
+  const int S = split_of(total);
   const int items = total * S;
-  // Stage size follows the tile this launch uses (A box of 128 rows or less, bn weight rows); the freed
-  // shared memory becomes more stages, i.e. more bytes in flight per SM when the launch streams weights.
+  // A pipeline stage holds two 64-wide k-blocks, each an A box of at most 128 rows (sized to the live rows) and
+  // the tile's weight rows; shared memory left over by small boxes becomes more stages, i.e. more bytes in
+  // flight per SM when the launch streams weights.
   const int a_rows_max = n >= 128 ? 128 : (n > 64 ? 128 : (n > 32 ? 64 : 32));
-  const int stage_bytes = ((a_rows_max + ((EPI == EPI_SWIGLU) ? ACC_COLS : bn)) * TK * 2 + 1023) & ~1023;
+  const int b_rows = (EPI == EPI_SWIGLU) ? ACC_COLS : bn;
+  const int sub_bytes = ((a_rows_max + b_rows) * TK * 2 + 1023) & ~1023;
+  const int stage_bytes = KSUB * sub_bytes;
   // the MMA always reads 128 rows of A: keep that read inside the allocation when the A box is smaller
   const int nst = min(ST_MAX, (ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2) / stage_bytes);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t it = 0;                                        // k-blocks issued so far (ring position)
+      uint32_t it = 0;                                        // stages issued so far (ring position)
       bool ok = true;
       for (int item = blockIdx.x; item < items && ok; item += G) {
         const int tile = item % total, part = item / total;
@@ -127,19 +145,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         const int m0 = (tile % MT) * TM, n0 = (tile / MT) * OUT_COLS;
         const int rows = n - m0;                              // live rows of this tile: load no more than needed
         const CUtensorMap* ma = rows <= 32 ? &tmA32 : (rows <= 64 ? &tmA64 : &tmA128);
-        const uint32_t a_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2;
-        for (int kt = k0; kt < k1; ++kt, ++it) {
+        const uint32_t kb_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2 + (uint32_t)b_rows * TK * 2;
+        for (int kt = k0; kt < k1; kt += KSUB, ++it) {
           const int s = it % nst;
+          const int nsub = min(KSUB, k1 - kt);
           if (!mbar_wait(empty_bar(s), ((it / nst) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
-          const uint32_t sa = smem_base + s * stage_bytes, sb = sa + a_rows_max * TK * 2;
-          mbar_expect_tx(full_bar(s), a_bytes + (uint32_t)bn * TK * 2);
-          tma_load_2d(sa, ma, kt * TK, m0, full_bar(s));
-          if (bn == 64) {
-            tma_load_2d(sb, &tmB64, kt * TK, n0, full_bar(s));
-          } else {
-            tma_load_2d(sb, &tmB, kt * TK, n0, full_bar(s));
-            if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kt * TK, n0, full_bar(s));
-            else if (bn == 256) tma_load_2d(sb + 128 * TK * 2, &tmB, kt * TK, n0 + 128, full_bar(s));
+          mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
+#pragma unroll
+          for (int u = 0; u < KSUB; ++u) {
+            if (u < nsub) {
+              const uint32_t sa = smem_base + s * stage_bytes + u * sub_bytes, sb = sa + a_rows_max * TK * 2;
+              const int kc = (kt + u) * TK;
+              tma_load_2d(sa, ma, kc, m0, full_bar(s));
+              if (bn == 64) {
+                tma_load_2d(sb, &tmB64, kc, n0, full_bar(s));
+              } else {
+                tma_load_2d(sb, &tmB, kc, n0, full_bar(s));
+                if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kc, n0, full_bar(s));
+                else if (bn == 256) tma_load_2d(sb + 128 * TK * 2, &tmB, kc, n0 + 128, full_bar(s));
+              }
+            }
           }
         }
       }
@@ -156,25 +181,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc(bn);
-      uint32_t it = 0, tcount = 0;
+      uint32_t tcount = 0;
       bool ok = true;
+      const uint64_t desc0 = smem_desc_sw128(smem_base);     // A operand of stage 0, k-block 0
+      const uint32_t b_off = (uint32_t)(a_rows_max * TK * 2) >> 4, sub_step = (uint32_t)sub_bytes >> 4;
+      int st = 0; uint32_t ph = 0;                           // ring position of the next stage
       for (int item = blockIdx.x; item < items && ok; item += G, ++tcount) {
         const int part = item / total;
-        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
+        const int nk = (part + 1) * KT / S - part * KT / S;
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 4)) { ok = false; break; }
-        tc_fence_after();
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
-        for (int kt = k0; kt < k1; ++kt, ++it) {
-          const int s = it % nst;
-          if (!mbar_wait(full_bar(s), (it / nst) & 1, abortp, status, 2)) { ok = false; break; }
+        for (int j = 0; j < nk; j += KSUB) {
+          const int nsub = min(KSUB, nk - j);
+          if (!mbar_wait(full_bar(st), ph, abortp, status, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + s * stage_bytes, sb = sa + a_rows_max * TK * 2;
-          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+          const uint64_t adesc = desc0 + (uint64_t)(st * (stage_bytes >> 4)), bdesc = adesc + b_off;
 #pragma unroll
-          for (int k = 0; k < TK / 16; ++k)                   // +32 bytes per K=16 slice inside the swizzle atom
-            umma_ss(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, ((kt - k0) | k) != 0);
-          umma_commit(empty_bar(s));                          // stage reusable once these MMAs have read it
+          for (int u = 0; u < KSUB; ++u) {
+            if (u < nsub) {
+#pragma unroll
+              for (int k = 0; k < TK / 16; ++k)               // +32 bytes per K=16 slice inside the swizzle atom
+                umma_ss(tacc, adesc + u * sub_step + 2 * k, bdesc + u * sub_step + 2 * k, idesc, (j | u | k) != 0);
+            }
+          }
+          umma_commit(empty_bar(st));                         // stage reusable once these MMAs have read it
+          if (++st == nst) { st = 0; ph ^= 1; }
         }
         if (ok) umma_commit(acc_full(buf));                   // accumulator complete
       }
@@ -191,7 +223,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       const int m0 = (tile % MT) * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
-      if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 3)) break;
+      // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
+      const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 3));
+      if (S > 1) {
+        // ... and, where the four warps meet at named barriers below, for all of them together
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*abortp) break;
+      } else if (!got) {
+        break;
+      }
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       bool reduce = false;
@@ -231,21 +271,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
           tmem_ld32(tbase + col, v);
           tmem_ld_wait();
         } else {
-          float4 t[4][8];
           const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + (size_t)(tile * S) * (TM * ACC_COLS)) +
                              (size_t)(col >> 2) * TM + lrow;
+          float4 acc[8];
 #pragma unroll
-          for (int c2 = 0; c2 < 4; ++c2)
+          for (int q = 0; q < 8; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+          for (int c0 = 0; c0 < S; c0 += 4) {                 // parts are added in part order, four loads in flight
+            float4 t[4][8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-              t[c2][q] = (c2 < S && row_ok) ? __ldcg(sp + (size_t)c2 * (TM * ACC_COLS / 4) + (size_t)q * TM) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c2 = 0; c2 < 4; ++c2)
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                t[c2][q] = (c0 + c2 < S && row_ok) ? __ldcg(sp + (size_t)(c0 + c2) * (TM * ACC_COLS / 4) + (size_t)q * TM) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int c2 = 0; c2 < 4; ++c2)
+#pragma unroll
+              for (int q = 0; q < 8; ++q) { acc[q].x += t[c2][q].x; acc[q].y += t[c2][q].y; acc[q].z += t[c2][q].z; acc[q].w += t[c2][q].w; }
+          }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            float4 acc = t[0][q];
-#pragma unroll
-            for (int c2 = 1; c2 < 4; ++c2) { acc.x += t[c2][q].x; acc.y += t[c2][q].y; acc.z += t[c2][q].z; acc.w += t[c2][q].w; }
-            v[4 * q] = __float_as_uint(acc.x); v[4 * q + 1] = __float_as_uint(acc.y);
-            v[4 * q + 2] = __float_as_uint(acc.z); v[4 * q + 3] = __float_as_uint(acc.w);
+            v[4 * q] = __float_as_uint(acc[q].x); v[4 * q + 1] = __float_as_uint(acc[q].y);
+            v[4 * q + 2] = __float_as_uint(acc[q].z); v[4 * q + 3] = __float_as_uint(acc[q].w);
           }
         }
       };
@@ -255,7 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS);
       } else if (EPI == EPI_SWIGLU) {
-        epilogue_swiglu(load_chunk, g, ew, n0);
+        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS);
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
         for (int half = 0; half < bn / 128; ++half) {         // statistics are kept per 128 columns

@@ -9,6 +9,13 @@
 // one-SM kernel.  TMA loads of both CTAs signal the even CTA's mbarrier (cta_group::2 form, no multicast
 // load); stage release and accumulator hand-over reach both CTAs through multicast tcgen05.commit.
 // Persistent: cluster c works on pair-tiles c, c + #clusters, ... with the row tile fastest.
+//
+// One thread issues every tcgen05.mma of a pair, and each step of its loop costs issue latency that does not
+// shrink with the tile: about 115 clocks for the full-barrier test, 58 per MMA and 95 for the commit (measured
+// with clock stamps on B200).  With one 64-wide k-block per pipeline stage that is ~560 clocks against the 512
+// clocks four M256 x N256 x K16 instructions run, so the tensor pipe waited on the issuing thread.  A stage
+// therefore holds two k-blocks (K = 128): eight MMAs per barrier round-trip, ~750 clocks of issue for 1024
+// clocks of tensor work.
 #include "common.cuh"
 #include "epilogue_tiles.cuh"
 #include "sm100_ptx.cuh"
@@ -20,8 +27,10 @@ constexpr int TM = 128, TK = 64;
 constexpr int TC_THREADS = 192;
 constexpr int A_BYTES = TM * TK * 2;             // 16 KB: this CTA's rows
 constexpr int BH_BYTES = 128 * TK * 2;           // 16 KB: this CTA's half of the weight tile
-constexpr int STAGE2 = A_BYTES + BH_BYTES;       // 32 KB per CTA and stage
-constexpr int ST2 = 6;
+constexpr int SUB2 = A_BYTES + BH_BYTES;         // 32 KB per CTA and k-block
+constexpr int KSUB = 2;                          // k-blocks per pipeline stage
+constexpr int STAGE2 = KSUB * SUB2;              // 64 KB per CTA and stage
+constexpr int ST2 = 3;
 constexpr int ACC_COLS = 256;
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;      // clears the CTA-rank bit of a shared::cluster address: the even CTA
 
@@ -110,23 +119,25 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n = *g.n_rows;
   const int MT = (max(n, 0) + 2 * TM - 1) / (2 * TM);
-  // Accumulator width: 256 columns, halved (to 128, then 64) while the narrower tiling fills the last
-  // wave of clusters so much better that it outweighs the far less efficient narrow MMA (measured factor ~0.6).
-  int bn = ACC_COLS;
   const int KT = g.K / TK;
   const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
-  const int t256 = MT * ((g.N + (EPI == EPI_SWIGLU ? 128 : 256) - 1) / (EPI == EPI_SWIGLU ? 128 : 256));
-  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;   // split-K beats narrow tiles
-  if ((EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split) {
-    while (bn > 64) {
-      const int t_wide = MT * ((g.N + bn - 1) / bn), t_narrow = MT * ((g.N + bn / 2 - 1) / (bn / 2));
-      if (t_wide == 0) break;
-      const float e_wide = (float)t_wide / (float)(((t_wide + ncl - 1) / ncl) * ncl);
-      const float e_narrow = (float)t_narrow / (float)(((t_narrow + ncl - 1) / ncl) * ncl);
-      if (e_narrow * 0.6f > e_wide) bn >>= 1; else break;
+  // Accumulator width of this launch.  With the issue latency out of the way a tile's time follows the bytes
+  // each SM pulls from L2 per k-block (its 128 rows of A plus its half of the weight rows; about 90 GB/s per SM
+  // measured), so a tile of half the width costs about 0.75 of a full one and a quarter-width one 0.73 (there
+  // the issuing thread is the limit again).  Narrow tiles only pay when they fill the launch's waves of
+  // clusters that much better; split-K (below) is preferred when few tiles are live.
+  int bn = ACC_COLS;
+  auto waves = [&](int out_cols) { const int t = MT * ((g.N + out_cols - 1) / out_cols); return (t + ncl - 1) / ncl; };
+  if (MT > 0 && (EPI == EPI_STORE || EPI == EPI_RESIDUAL)) {
+    const int t256 = MT * ((g.N + 255) / 256);
+    const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;
+    if (!will_split) {
+      float best = (float)waves(256);
+      if ((float)waves(128) * 0.75f < best) { best = (float)waves(128) * 0.75f; bn = 128; }
+      if ((float)waves(64) * 0.73f < best) { bn = 64; }
     }
   }
-  const int OUT_COLS = (EPI == EPI_SWIGLU) ? 128 : bn;       // output columns per pair-tile
+  const int OUT_COLS = (EPI == EPI_SWIGLU) ? bn / 2 : bn;    // output columns per pair-tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
   const int total = MT * NT;                                 // 0 when no row is live: every role loop is empty
   // Split-K when there are fewer pair-tiles than clusters: K is cut into S equal parts, one (tile, part)
@@ -136,25 +147,33 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   if (sk_ok && total > 0 && total < ncl && 2 * total <= g.sk_max_tiles)
     S = max(1, min(min(ncl / total, KT / 8), 4));
   const int items = total * S;
+  const int b_box_rows = bn / 2;                             // weight rows this CTA brings in per k-block
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0;                                        // stages issued so far (ring position)
       bool ok = true;
+      const uint32_t kb_bytes = 2 * (A_BYTES + (uint32_t)b_box_rows * TK * 2);   // both CTAs' boxes of one k-block
+      const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
       for (int item = cl; item < items && ok; item += ncl) {
         const int tile = item % total, part = item / total;
         const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
-        const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
         const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
-        for (int kt = k0; kt < k1; ++kt, ++it) {
+        for (int kt = k0; kt < k1; kt += KSUB, ++it) {
           const int s = it % ST2;
+          const int nsub = min(KSUB, k1 - kt);
           if (!mbar_wait(empty_bar(s), ((it / ST2) & 1) ^ 1, abortp, status, 31)) { ok = false; break; }
-          const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
-          if (leader) mbar_expect_tx(full_bar(s), 2 * (A_BYTES + (uint32_t)(bn / 2) * TK * 2));   // both CTAs' boxes
-          tma_load_2d_pair(sa, &tmA, kt * TK, m0, full_bar(s));
-          tma_load_2d_pair(sb, mb, kt * TK, brow, full_bar(s));
+          if (leader) mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
+#pragma unroll
+          for (int u = 0; u < KSUB; ++u) {
+            if (u < nsub) {
+              const uint32_t sa = smem_base + s * STAGE2 + u * SUB2, sb = sa + A_BYTES;
+              tma_load_2d_pair(sa, &tmA, (kt + u) * TK, m0, full_bar(s));
+              tma_load_2d_pair(sb, mb, (kt + u) * TK, brow, full_bar(s));
+            }
+          }
         }
       }
       if (*abortp && leader) {
@@ -168,26 +187,32 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (even CTA only)
     if (lane == 0 && leader) {
-      uint32_t it = 0, tcount = 0;
+      uint32_t tcount = 0;
       bool ok = true;
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((256u >> 4) << 24);
+      const uint64_t desc0 = smem_desc_sw128(smem_base);     // A operand of stage 0, k-block 0
+      int st = 0; uint32_t ph = 0;                           // ring position of the next stage
       for (int item = cl; item < items && ok; item += ncl, ++tcount) {
         const int part = item / total;
-        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
+        const int nk = (part + 1) * KT / S - part * KT / S;
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 34)) { ok = false; break; }
-        tc_fence_after();
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
-        for (int kt = k0; kt < k1; ++kt, ++it) {
-          const int s = it % ST2;
-          if (!mbar_wait(full_bar(s), (it / ST2) & 1, abortp, status, 32)) { ok = false; break; }
+        for (int j = 0; j < nk; j += KSUB) {
+          const int nsub = min(KSUB, nk - j);
+          if (!mbar_wait(full_bar(st), ph, abortp, status, 32)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE2, sb = sa + A_BYTES;
-          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+          const uint64_t adesc = desc0 + (uint64_t)(st * (STAGE2 >> 4)), bdesc = adesc + (A_BYTES >> 4);
 #pragma unroll
-          for (int k = 0; k < TK / 16; ++k)
-            umma2_bf16(tacc, adesc + 2 * k, bdesc + 2 * k, idesc, ((kt - k0) | k) != 0);
-          umma2_commit_both(empty_bar(s));                    // both CTAs may refill this stage
+          for (int u = 0; u < KSUB; ++u) {
+            if (u < nsub) {
+#pragma unroll
+              for (int k = 0; k < TK / 16; ++k)               // +32 bytes per K=16 slice inside the swizzle atom
+                umma2_bf16(tacc, adesc + u * (SUB2 >> 4) + 2 * k, bdesc + u * (SUB2 >> 4) + 2 * k, idesc, (j | u | k) != 0);
+            }
+          }
+          umma2_commit_both(empty_bar(st));                   // both CTAs may refill this stage
+          if (++st == ST2) { st = 0; ph ^= 1; }
         }
         if (ok) umma2_commit_both(acc_full(buf));             // both CTAs' epilogues may read their rows
       }
@@ -204,13 +229,21 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
-      if (!mbar_wait(acc_full(buf), use & 1, abortp, status, 33)) break;
+      // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
+      const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 33));
+      if (S > 1) {
+        // ... and, where the four warps meet at named barriers below, for all of them together
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*abortp) break;
+      } else if (!got) {
+        break;
+      }
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       bool reduce = false;
       const size_t slot_floats = (size_t)TM * ACC_COLS;
       if (S > 1) {
-        const int acc_cols = (EPI == EPI_SWIGLU) ? ACC_COLS : bn;
+        const int acc_cols = bn;
         float4* mine = reinterpret_cast<float4*>(g.sk_partials + ((size_t)(tile * S + part) * 2 + rank) * slot_floats);
 #pragma unroll 1
         for (int c = 0; c < acc_cols / 32; ++c) {
@@ -269,7 +302,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
         epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS);
       } else if (EPI == EPI_SWIGLU) {
-        epilogue_swiglu(load_chunk, g, ew, n0);
+        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS);
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {         // statistics are kept per 128 columns
