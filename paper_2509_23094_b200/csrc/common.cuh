@@ -68,6 +68,7 @@ struct SelectArgs {
   float* key; int32_t* sel_idx; int32_t* row_seq; int32_t* row_off; int32_t* lm_rows; int32_t* lm_off;
   int32_t* slot_of_pos;
   int32_t* rank_s; int32_t* rank_lm; int32_t* n_b; int32_t* nm_b;   // scratch [B][L],[B][L],[B],[B]
+  int32_t* n_host;                               // optional: device-visible address of a host word that receives the total row count
 };
 int launch_select(const SelectArgs& a, cudaStream_t st);
 // Fills tab[0..len) with floor(exp(-r^2/(2 sigma^2)) * 2^30 + 0.5); returns the first r whose entry is 0 (or len).

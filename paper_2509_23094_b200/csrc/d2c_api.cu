@@ -114,9 +114,16 @@ struct d2c_ctx {
   cudaStream_t stream;
   Buffers buf;
   int phi_len;
-  // Selected-row count of an earlier step, copied to pinned host memory at the end of every step and read
-  // without synchronising: only a hint for choosing between GEMM kernels (both are correct for any count).
-  int32_t* n_hint = nullptr;
+  // Selected-row count of the previous step, which chooses between the GEMM kernels (both are correct for any
+  // count, but they add fp32 partial sums in different orders).  The selection kernel writes the count into one
+  // of two words of mapped host memory; the next step waits for the event recorded behind that kernel before it
+  // reads the word, so the choice depends on the step sequence only, never on how far the host runs ahead.
+  int32_t* hint_host[2] = {nullptr, nullptr};
+  int32_t* hint_dev[2] = {nullptr, nullptr};
+  cudaEvent_t ev_hint[2] = {nullptr, nullptr};
+  long long hint_step[2] = {-1, -1};     // step number whose count the word holds
+  long long step_no = 0;
+  bool few_rows = false;                 // this step's regime: at most 128 rows expected
   // d2c_step_host: the device-to-host copy of the hidden rows runs on its own stream, ordered after the
   // last layer by an event, so that it overlaps the LM head and the rollout
   cudaStream_t copy_stream = nullptr;
@@ -184,7 +191,7 @@ static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->run);
   // The LM head runs on few rows and is bound by the weight stream: the one-SM kernel sizes its A boxes to the
   // live rows, a pair would load a second, empty row tile.
-  const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;   // weight-streaming regime
+  const bool few_rows = ctx->few_rows;                      // weight-streaming regime
   if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && !few_rows && gemm_tc2_supported(g))
   {
     GemmArgs g2 = g;
@@ -239,8 +246,21 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
   }
   ctx->g_final = (const bf16*)w->g_final; ctx->w_lm = (const bf16*)w->w_lm;
   carve(*cfg, workspace, &ctx->buf);
-  if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->n_hint), sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess) *ctx->n_hint = 1 << 30;
-  else { ctx->n_hint = nullptr; (void)cudaGetLastError(); }
+  {
+    bool ok = cudaHostAlloc(reinterpret_cast<void**>(&ctx->hint_host[0]), 2 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
+    if (ok) {
+      ctx->hint_host[1] = ctx->hint_host[0] + 1;
+      ctx->hint_host[0][0] = ctx->hint_host[0][1] = 1 << 30;
+      ok = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->hint_dev[0]), ctx->hint_host[0], 0) == cudaSuccess;
+      ctx->hint_dev[1] = ctx->hint_dev[0] + 1;
+      for (int i = 0; i < 2 && ok; ++i) ok = cudaEventCreateWithFlags(&ctx->ev_hint[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) {                                               // the step then always takes the many-row kernels
+      for (int i = 0; i < 2; ++i) if (ctx->ev_hint[i]) { cudaEventDestroy(ctx->ev_hint[i]); ctx->ev_hint[i] = nullptr; }
+      if (ctx->hint_host[0]) cudaFreeHost(ctx->hint_host[0]);
+      ctx->hint_host[0] = ctx->hint_host[1] = nullptr; (void)cudaGetLastError();
+    }
+  }
   if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->layers_done, cudaEventDisableTiming) != cudaSuccess) {
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -275,7 +295,8 @@ int d2c_create(const d2c_config* cfg, const d2c_weights* w, void* workspace, siz
 int d2c_destroy(d2c_ctx* ctx) {
   if (!ctx) return D2C_EINVAL;
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
-  if (ctx->n_hint) cudaFreeHost(ctx->n_hint);
+  for (int i = 0; i < 2; ++i) if (ctx->ev_hint[i]) cudaEventDestroy(ctx->ev_hint[i]);
+  if (ctx->hint_host[0]) cudaFreeHost(ctx->hint_host[0]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->layers_done) cudaEventDestroy(ctx->layers_done);
   destroy_overlap(ctx);
@@ -335,7 +356,22 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   // that follow: in the weight-streaming regime (few rows: short CTAs, GEMMs bound by HBM) and for a single
   // layer (it then overlaps the LM head).  Otherwise a statically scheduled GEMM whose CTAs start late behind
   // side-stream CTAs loses more than the overlap gains (measured at 488 rows x 32 layers: +5 %).
-  const bool few_rows = ctx->n_hint && *reinterpret_cast<volatile int32_t*>(ctx->n_hint) <= 128;
+  // regime of this step: the row count of the previous step, read behind that step's selection kernel
+  bool capturing = false;
+  {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(ctx->stream, &cs) != cudaSuccess) { (void)cudaGetLastError(); capturing = true; }
+    else capturing = cs != cudaStreamCaptureStatusNone;
+  }
+  const bool track = ctx->hint_host[0] != nullptr && !capturing;
+  const int slot = (int)(ctx->step_no & 1), prev = slot ^ 1;
+  int expect_rows = 1 << 30;
+  if (track && ctx->hint_step[prev] == ctx->step_no - 1) {
+    D2C_TRY(ctx, cu(cudaEventSynchronize(ctx->ev_hint[prev])));
+    expect_rows = *reinterpret_cast<volatile int32_t*>(ctx->hint_host[prev]);
+  }
+  ctx->few_rows = expect_rows <= 128;
+  const bool few_rows = ctx->few_rows;
   const bool abar_aside = overlap && (c.n_layers == 1 || few_rows);
   bool abar_pending = false, rollout_done = false;
   // Eq. 6-9 for the next step's stage 2: enqueued right after the last probabilities pass it needs
@@ -356,8 +392,14 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   s.stage2_candidates = c.stage2_candidates; s.block_lo = a->block_lo; s.block_hi = a->block_hi; s.phi_q30 = b.phi; s.phi_len = ctx->phi_len < L ? ctx->phi_len : L;
   s.key = b.key; s.sel_idx = b.sel_idx; s.row_seq = b.row_seq; s.row_off = b.row_off; s.lm_rows = b.lm_rows;
   s.lm_off = b.lm_off; s.slot_of_pos = b.slot_of_pos; s.rank_s = b.rank_s; s.rank_lm = b.rank_lm; s.n_b = b.n_b; s.nm_b = b.nm_b;
+  s.n_host = track ? ctx->hint_dev[slot] : nullptr;
   D2C_TRY(ctx, mark(ctx, PH_SELECT));
   D2C_TRY(ctx, launch_select(s, st));
+  if (track) {
+    D2C_TRY(ctx, cu(cudaEventRecord(ctx->ev_hint[slot], st)));
+    ctx->hint_step[slot] = ctx->step_no;
+  }
+  ctx->step_no++;
   const int32_t* n_rows = b.row_off + B;
   const int32_t* n_lm = b.lm_off + B;
 
@@ -468,10 +510,6 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   }
   if (out && out->row_off) {
     cudaError_t e = cudaMemcpyAsync(out->row_off, b.row_off, (size_t)(B + 1) * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
-    if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
-  }
-  if (ctx->n_hint) {
-    cudaError_t e = cudaMemcpyAsync(ctx->n_hint, b.row_off + B, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
   }
   D2C_TRY(ctx, mark(ctx, -1));

@@ -14,6 +14,7 @@
 namespace d2c {
 
 static constexpr int kSelThreads = 1024;
+static constexpr int kPhiMax = 512;              // phi entries kept in shared memory; a wider window reads the rest from global memory
 enum : uint8_t { F_SEL = 1, F_MSTAR = 2 };
 
 // Descending bitonic sort of n 64-bit words in shared memory by the whole block.  Pair p of a stage exchanges
@@ -83,6 +84,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
   __shared__ uint64_t s_total64;
   __shared__ int warp_buf32[32];
   __shared__ int s_total32, s_cnt, s_take;
+  __shared__ uint32_t s_phi[kPhiMax];                          // the non-zero head of the phi table (window +-65 at sigma 10)
 
   const int b = blockIdx.x, L = a.seq_len, tid = threadIdx.x;
   const uint8_t* mask = a.mask + (size_t)b * L;
@@ -93,6 +95,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
   // stage 1 may be confined to one block of positions (semi-autoregressive decoding); whole sequence otherwise
   const int blk_lo = a.block_hi > a.block_lo ? a.block_lo : 0, blk_hi = a.block_hi > a.block_lo ? a.block_hi : L;
   for (int i = tid; i < L; i += kSelThreads) { smask[i] = mask[i] ? 1 : 0; flags[i] = 0; }
+  for (int r = tid; r < min(a.phi_len, kPhiMax); r += kSelThreads) s_phi[r] = a.phi_q30[r];
   if (tid == 0) { s_cnt = 0; }
   __syncthreads();
 
@@ -113,7 +116,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
               int known = 0;
               if (lo >= 0) known += 1 - smask[lo];
               if (hi < L) known += 1 - smask[hi];
-              dq += (unsigned long long)a.phi_q30[r] * (unsigned)known;
+              dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * (unsigned)known;
             }
             const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;   // * 2^-30, exact
             key = clean_score(__fmul_rn(D, conf[i]));
@@ -192,7 +195,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
             int known = 0;
             if (lo >= 0) known += 1 - smask[lo];
             if (hi < L) known += 1 - smask[hi];
-            dq += (unsigned long long)a.phi_q30[r] * (unsigned)known;
+            dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * (unsigned)known;
           }
           const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;   // * 2^-30, exact
           key = clean_score(__fmul_rn(D, conf[i]));
@@ -299,8 +302,22 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P
       }
       a.rank_s[(size_t)b * L + j] = rs;
       a.rank_lm[(size_t)b * L + j] = rl;
+      if (a.batch == 1) {
+        // one sequence: its ranks are the global row numbers, so the second kernel's work is done here
+        if (rs >= 0) {
+          a.sel_idx[rs] = j; a.row_seq[rs] = 0;
+          if (rl >= 0) a.lm_rows[rl] = rs;
+        }
+        a.slot_of_pos[j] = rs;
+      }
     }
     if (tid == 0) { a.n_b[b] = s_total32 & 0xFFFF; a.nm_b[b] = s_total32 >> 16; }
+    if (a.batch == 1) {
+      if (tid == 0) {
+        a.row_off[0] = 0; a.lm_off[0] = 0; a.row_off[1] = s_total32 & 0xFFFF; a.lm_off[1] = s_total32 >> 16;
+        if (a.n_host) *a.n_host = s_total32 & 0xFFFF;
+      }
+    }
   }
 }
 
@@ -312,7 +329,10 @@ __global__ void __launch_bounds__(256) select_finalize_kernel(SelectArgs a) {
   for (int bb = 0; bb < b; ++bb) { off += a.n_b[bb]; lmoff += a.nm_b[bb]; }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     a.row_off[b] = off; a.lm_off[b] = lmoff;
-    if (b == a.batch - 1) { a.row_off[a.batch] = off + a.n_b[b]; a.lm_off[a.batch] = lmoff + a.nm_b[b]; }
+    if (b == a.batch - 1) {
+      a.row_off[a.batch] = off + a.n_b[b]; a.lm_off[a.batch] = lmoff + a.nm_b[b];
+      if (a.n_host) *a.n_host = off + a.n_b[b];
+    }
   }
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < L; j += gridDim.x * blockDim.x) {
     const int rs = a.rank_s[(size_t)b * L + j];
@@ -341,8 +361,10 @@ int launch_select(const SelectArgs& a, cudaStream_t st) {
     attr_set = true;
   }
   D2C_LAUNCH((select_kernel), a.batch, kSelThreads, smem, st, a, P2);
-  dim3 grid(ceil_div(a.seq_len, 256), a.batch);
-  D2C_LAUNCH((select_finalize_kernel), grid, 256, 0, st, a);
+  if (a.batch > 1) {
+    dim3 grid(ceil_div(a.seq_len, 256), a.batch);
+    D2C_LAUNCH((select_finalize_kernel), grid, 256, 0, st, a);
+  }
   return D2C_OK;
 }
 
