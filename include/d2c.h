@@ -178,11 +178,14 @@ typedef struct {
   int32_t* status;      /* [4] device status word: [0] error code, [1] where                         */
 } d2c_state;
 /* The per-position vectors (conf, pred, c, key) are indexed [b*seq_len + pos] with the batch and
- * seq_len of the d2c_step calls; a context is used with one (batch, seq_len) from its first step on.
+ * seq_len of the d2c_step calls; a context is used with one (batch, seq_len) from its first step on
+ * (d2c_step and d2c_commit return D2C_EINVAL for any other pair).
  * abar: row r of layer l is at abar + l*max_batch*max_seq*max_seq + r*seq_len. */
 int d2c_state_ptrs(d2c_ctx* ctx, d2c_state* out);
 
-/* Synchronises the stream and returns the device status word's error code. */
+/* Synchronises the stream and returns the device status word's error code (D2C_OK, or what a kernel's
+ * bounded wait recorded: D2C_ETIMEOUT with the wait's site number in the error text).  The word is sticky:
+ * it keeps the first error until the caller writes zeros to status[0..3]. */
 int d2c_sync_status(d2c_ctx* ctx);
 
 /* Per-phase timing of d2c_step.  While enabled, d2c_step records one CUDA event at every phase
@@ -216,7 +219,9 @@ size_t d2c_op_select_scratch_bytes(int32_t batch, int32_t seq_len);
  * override_key / forced / forced_off optional (NULL).  Outputs: key [batch][seq_len];
  * sel_idx [batch*seq_len]; row_off [batch+1]; lm_rows [batch*seq_len] and lm_off
  * [batch+1]: global row numbers of the selected rows that are masked;
- * slot_of_pos [batch][seq_len]: row number of a selected position, else -1. */
+ * slot_of_pos [batch][seq_len]: row number of a selected position, else -1.
+ * Unlike the other stand-alone kernels this call synchronises `cuda_stream` once before it enqueues its
+ * kernels: it builds the phi table of Eq. 3 in host memory and copies it into the scratch first. */
 int d2c_op_select(const uint8_t* mask, const float* conf, const float* c, const float* override_key,
                   const int32_t* forced, const int32_t* forced_off, int32_t batch, int32_t seq_len,
                   int32_t k, float p, float sigma, int32_t stage2_candidates,
@@ -263,6 +268,15 @@ size_t d2c_op_rollout_scratch_bytes(int32_t batch, int32_t seq_len);
 int d2c_op_rollout(const float* abar, size_t layer_stride, int32_t n_layers, const int32_t* sel_idx,
                    const int32_t* row_off, int32_t batch, int32_t seq_len, float* c,
                    void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+/* The library's bounded device-side wait, on its own.  Every pipeline wait of the tcgen05 kernels (on an
+ * mbarrier that a TMA copy or a tensor-core commit completes) gives up after a cycle limit, records
+ * D2C_ETIMEOUT in status[0] and the number of the wait that ran out in status[1], and lets the kernel drain
+ * and return; d2c_sync_status then reports it.  This entry launches one small CTA that waits, with the given
+ * limit (1e3 .. 2e9 SM clocks), on a barrier nothing arrives on: it returns after about that many clocks and
+ * leaves status = {D2C_ETIMEOUT, 99, ...}.  status: device int32[4], zeroed by the caller.  It exists so that
+ * the error path of section "Conventions" can be exercised without a fault; it has no counterpart in the paper. */
+int d2c_op_wait_probe(int32_t* status, int64_t limit_cycles, void* cuda_stream);
 
 /* d2c_op_rollout without a scratch argument.  (The paper has no counterpart for this entry point; it
  * exists for integration reasons only.)  It serves callers that cannot get device memory at the time

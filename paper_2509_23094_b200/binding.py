@@ -21,7 +21,7 @@ D2C_OK, D2C_EINVAL, D2C_ESHAPE, D2C_ECAPACITY, D2C_ECUDA, D2C_ETIMEOUT = 0, -1, 
 SYMBOLS = ["d2c_workspace_bytes", "d2c_create", "d2c_step", "d2c_step_host", "d2c_commit", "d2c_state_ptrs",
            "d2c_sync_status", "d2c_last_error", "d2c_destroy", "d2c_profile", "d2c_profile_read", "d2c_phase_name", "d2c_op_select_scratch_bytes", "d2c_op_select",
            "d2c_op_gemm", "d2c_op_attention", "d2c_op_lm_head_scratch_bytes", "d2c_op_lm_head",
-           "d2c_op_rollout_scratch_bytes", "d2c_op_rollout", "d2c_op_rollout_static"]
+           "d2c_op_rollout_scratch_bytes", "d2c_op_rollout", "d2c_op_rollout_static", "d2c_op_wait_probe"]
 
 
 class D2cError(RuntimeError):
@@ -354,3 +354,11 @@ def d2c_op_rollout_static(abar, sel_idx, row_off, batch, seq_len, c=None):
     _check(load().d2c_op_rollout_static(_ptr(abar), abar.stride(0), abar.shape[0], _ptr(sel_idx), _ptr(row_off), batch,
                                         seq_len, _ptr(c), _stream_ptr()))
     return c
+
+
+def d2c_op_wait_probe(status: torch.Tensor, limit_cycles: int = 100000):
+    """Runs the library's bounded device-side wait on a barrier nothing arrives on; status: int32[4] on the device."""
+    assert status.dtype == torch.int32 and status.numel() >= 4
+    lib = load()
+    lib.d2c_op_wait_probe.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+    _check(lib.d2c_op_wait_probe(_ptr(status), int(limit_cycles), _stream_ptr()))

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2c.so")
 SOURCES = ["d2c_api.cu", "ops_api.cu", "select.cu", "rows.cu", "gemm_mma.cu", "gemm_tc.cu", "gemm_tc2.cu", "attention.cu", "attention_tc.cu",
-           "lmhead.cu", "rollout.cu", "commit.cu", "rollout_static.cu"]
+           "lmhead.cu", "rollout.cu", "commit.cu", "rollout_static.cu", "wait_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O3"]
 # The selection and commit kernels decide indices from fp32 products and must round exactly like

@@ -250,11 +250,10 @@ __global__ void __launch_bounds__(ATHREADS) attn_abar_kernel(AttnArgs a) {
 template <int DH>
 int launch_dh(const AttnArgs& a, cudaStream_t st) {
   const int smem_fwd = QT * DH * 2 + 4 * KT * DH * 2, smem_ab = 4 * KT * DH * 2;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(attn_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_fwd));
     D2C_CUDA_OK(cudaFuncSetAttribute(attn_abar_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_ab));
-    attr_set = true;
   }
   const int qtiles = ceil_div(a.max_rows_per_seq, QT);
   if (a.which != 2) {

@@ -510,11 +510,10 @@ bool attention_tc_supported(const AttnArgs& a) {
 
 int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   const int smem_fwd = 6 * TILE_BYTES + 1024, smem_ab = 2 * ABS * TILE_BYTES + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_fwd));
     D2C_CUDA_OK(cudaFuncSetAttribute(attn_abar_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_ab));
-    attr_set = true;
   }
   CUtensorMap tmQ, tmK, tmV;
   const uint64_t kv_cols = (uint64_t)a.hkv * a.dh, kv_rows = (uint64_t)a.batch * a.cache_seq;
@@ -522,8 +521,7 @@ int launch_attention_tc(const AttnArgs& a, cudaStream_t st, int* status) {
   if (rc == D2C_OK) rc = make_bf16_map(&tmK, a.kc, kv_rows, kv_cols, kv_cols, 128);
   if (rc == D2C_OK) rc = make_bf16_map(&tmV, a.vc, kv_rows, kv_cols, kv_cols, 128);
   if (rc != D2C_OK) return rc;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 148;
+  const int sms = sm_count_current();
   const int qtiles = ceil_div(a.max_rows_per_seq, AQ), ktiles = ceil_div(a.seq_len, AKEYS);
   // split the heads over several CTAs while the (row tile x key tile) grid leaves a quarter of the SMs idle
   int groups = 1;

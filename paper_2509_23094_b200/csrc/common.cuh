@@ -55,6 +55,23 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // After a kernel launch: checks the launch and counts it.
 #define D2C_LAUNCHED() do { D2C_CUDA_OK(cudaGetLastError()); d2c::count_launch(1); } while (0)
 
+// Per-device one-time set-up (function attributes, device properties): kernels' attributes belong to the
+// device they were set on, so the "done" flags are kept per device ordinal, for the device that is current.
+constexpr int kMaxDevices = 64;
+struct PerDevice {
+  bool done[kMaxDevices] = {};
+  // true the first time it is called with this device current (and for ordinals beyond the table, every time)
+  bool first() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return true;
+    if (done[dev]) return false;
+    done[dev] = true;
+    return true;
+  }
+};
+// Multiprocessor count of the current device (looked up once per device).
+int sm_count_current();
+
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

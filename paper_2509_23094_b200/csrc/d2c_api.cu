@@ -17,6 +17,16 @@ void set_global_error(const char* fmt, ...) {
 }
 const char* global_error() { return g_err; }
 
+int sm_count_current() {
+  static int count[kMaxDevices] = {};
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < kMaxDevices && count[dev] > 0) return count[dev];
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  if (dev >= 0 && dev < kMaxDevices) count[dev] = n;
+  return n;
+}
+
 static thread_local long long g_launches = 0;
 void count_launch(int n) { g_launches += n; }
 
@@ -124,6 +134,7 @@ struct d2c_ctx {
   long long hint_step[2] = {-1, -1};     // step number whose count the word holds
   long long step_no = 0;
   bool few_rows = false;                 // this step's regime: at most 128 rows expected
+  int used_batch = 0, used_seq = 0;      // the (batch, seq_len) of the first step: the per-position state is laid out for it
   // d2c_step_host: the device-to-host copy of the hidden rows runs on its own stream, ordered after the
   // last layer by an event, so that it overlaps the LM head and the rollout
   cudaStream_t copy_stream = nullptr;
@@ -336,6 +347,10 @@ static int check_step_args(d2c_ctx* ctx, const d2c_step_args* a) {
   if (a->k < 0) return fail(ctx, D2C_EINVAL, "d2c_step: k = %d is negative", a->k);
   if (isnan(a->p)) return fail(ctx, D2C_EINVAL, "d2c_step: p is NaN");
   if ((a->forced == nullptr) != (a->forced_off == nullptr)) return fail(ctx, D2C_EINVAL, "d2c_step: forced and forced_off must be given together");
+  if (ctx->used_batch == 0) { ctx->used_batch = a->batch; ctx->used_seq = a->seq_len; }
+  if (a->batch != ctx->used_batch || a->seq_len != ctx->used_seq)
+    return fail(ctx, D2C_EINVAL, "d2c_step: batch %d x seq_len %d differs from the %d x %d this context was first used with",
+                a->batch, a->seq_len, ctx->used_batch, ctx->used_seq);
   return D2C_OK;
 }
 
@@ -599,6 +614,8 @@ int d2c_commit(d2c_ctx* ctx, int32_t batch, int32_t seq_len, const void* embed_t
   if (batch < 1 || batch > ctx->cfg.max_batch || seq_len < 1 || seq_len > ctx->cfg.max_seq)
     return fail(ctx, D2C_ECAPACITY, "d2c_commit: batch %d x seq_len %d out of range", batch, seq_len);
   if (rule < 0 || rule > 2 || isnan(threshold)) return fail(ctx, D2C_EINVAL, "d2c_commit: rule %d / threshold", rule);
+  if (ctx->used_batch != 0 && (batch != ctx->used_batch || seq_len != ctx->used_seq))
+    return fail(ctx, D2C_EINVAL, "d2c_commit: batch %d x seq_len %d differs from the %d x %d of this context's steps", batch, seq_len, ctx->used_batch, ctx->used_seq);
   const Buffers& b = ctx->buf;
   D2C_TRY(ctx, launch_commit(batch, seq_len, ctx->cfg.d_model, rule, threshold, b.slot_of_pos, b.conf, b.pred, b.phi,
                              ctx->phi_len < seq_len ? ctx->phi_len : seq_len, (const bf16*)embed_table, (bf16*)h0, mask,

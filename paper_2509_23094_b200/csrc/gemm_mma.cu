@@ -224,10 +224,9 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_mma_kernel(GemmArgs g) {
 template <int EPI>
 int launch_one(const GemmArgs& g, cudaStream_t st) {
   const int smem = STAGES * STAGE_BYTES;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_mma_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_set = true;
   }
   const int n_tiles = EPI == EPI_SWIGLU ? ceil_div(g.N, 64) : ceil_div(g.N, BN);
   dim3 grid(n_tiles, ceil_div(g.max_rows, BM));

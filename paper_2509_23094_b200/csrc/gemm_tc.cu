@@ -358,23 +358,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   }
 }
 
-int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 template <int EPI>
 int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   const int smem = ST * STAGE_BYTES + 1024 + 4 * kEpiStageBytes;   // stage ring, alignment slack, epilogue staging
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_set = true;
   }
   CUtensorMap tmA128, tmA64, tmA32, tmB, tmB2, tmB64;
   int rc = make_bf16_map(&tmA128, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
@@ -387,7 +376,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   TcParams p{g, status};
   const int out_cols = EPI == EPI_SWIGLU ? 128 : (EPI == EPI_LMSTATS ? 128 : (EPI == EPI_QKV_ROPE ? (g.q_dh > 64 ? g.q_dh : 64) : 64));   // narrowest tile
   const long long tiles = (long long)ceil_div(g.max_rows, TM) * ceil_div(g.N, out_cols);
-  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  const int grid = (int)(tiles < sm_count_current() ? tiles : sm_count_current());
   D2C_LAUNCH((gemm_tc_kernel<EPI>), grid, TC_THREADS, smem, st, tmA128, tmA64, tmA32, tmB, tmB2, tmB64, p);
   return D2C_OK;
 }

@@ -359,23 +359,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
 }
 
-int sm_count2() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 template <int EPI>
 int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   const int smem = ST2 * STAGE2 + 1024 + 4 * kEpiStageBytes;   // stage ring, alignment slack, epilogue staging
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_set = true;
   }
   CUtensorMap tmA, tmB, tmB2, tmB64, tmB32;
   int rc = make_bf16_map(&tmA, g.A, (uint64_t)g.max_rows, (uint64_t)g.K, (uint64_t)g.lda, 128);
@@ -387,7 +376,7 @@ int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
   Tc2Params p{g, status};
   const int out_cols = (EPI == EPI_STORE || EPI == EPI_RESIDUAL) ? 64 : (EPI == EPI_SWIGLU ? 128 : 256);   // narrowest tile (QKV: 256)
   const long long tiles = (long long)ceil_div(g.max_rows, 2 * TM) * ceil_div(g.N, out_cols);
-  const int pairs = (int)(tiles < sm_count2() / 2 ? tiles : sm_count2() / 2);
+  const int pairs = (int)(tiles < sm_count_current() / 2 ? tiles : sm_count_current() / 2);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute attr[2];

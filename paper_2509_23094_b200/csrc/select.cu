@@ -355,10 +355,9 @@ int launch_select(const SelectArgs& a, cudaStream_t st) {
   int P2 = 32;
   while (P2 < a.seq_len) P2 <<= 1;
   const size_t smem = (size_t)P2 * 8 + 2 * (size_t)a.seq_len;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDevice attr_set;
+  if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8192 * 8 + 2 * 8192));
-    attr_set = true;
   }
   D2C_LAUNCH((select_kernel), a.batch, kSelThreads, smem, st, a, P2);
   if (a.batch > 1) {

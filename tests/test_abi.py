@@ -75,3 +75,6 @@ def test_ops_reject_bad_arguments_without_a_device(lib):
     assert lib.d2c_op_attention(None, 1, 0, None, None, None, 1, 1, 1, 1, 1, 64, None, None, None, 0, None) == binding.D2C_EINVAL
     assert lib.d2c_op_lm_head(None, None, None, 1, 64, 2, None, None, None, None, 0, None) == binding.D2C_EINVAL
     assert lib.d2c_op_rollout(None, 0, 1, None, None, 1, 1, None, None, 0, None) == binding.D2C_EINVAL
+    lib.d2c_op_wait_probe.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+    assert lib.d2c_op_wait_probe(None, 100000, None) == binding.D2C_EINVAL
+    assert lib.d2c_op_wait_probe(256, 10, None) == binding.D2C_EINVAL            # limit below 1e3 clocks
