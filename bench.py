@@ -9,7 +9,9 @@ workload is one LLaDA-8B-shaped layer at sequence length 1024 (prefill, then the
 step with k=32, p=0.9).  Prints one JSON line.
 
 The path does not shard (one model replica per GPU, no exchange step): with --gpus N every rank
-runs an independent replica and the line reports the aggregate.
+runs an independent replica and the line reports the aggregate.  Started without a launcher,
+`--gpus N` (N > 1) re-executes itself under `python -m torch.distributed.run` with N ranks on
+127.0.0.1; started by a launcher (WORLD_SIZE set) it takes its rank from the environment.
 """
 from __future__ import annotations
 
@@ -66,7 +68,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.0005)
 
     def start(self):
         try:
@@ -117,6 +119,35 @@ def algorithmic_work(shape, batch, L, n_b, n_m, rollout_layers):
     return flops, byts
 
 
+def profiled_traffic(kernel_tag, path=None):
+    """DRAM bytes (read + write) of one launch of a kernel, from the committed ncu summary of this workload:
+    the first block of profiles/gemm_tc2_kernel_llada1l_1024.txt whose header names `kernel_tag`.
+    Returns (bytes, source) or (None, reason)."""
+    path = path or os.path.join(ROOT, "profiles", "gemm_tc2_kernel_llada1l_1024.txt")
+    unit = {"Gbyte": 1e9, "Mbyte": 1e6, "Kbyte": 1e3, "byte": 1.0}
+    try:
+        lines = open(path).read().splitlines()
+    except OSError:
+        return None, "no committed ncu summary"
+    rd = wr = None
+    inside = False
+    for ln in lines:
+        if not ln.startswith(" "):
+            if inside and rd is not None and wr is not None:
+                break
+            inside = kernel_tag in ln
+            continue
+        if inside:
+            f = ln.split()
+            if len(f) >= 3 and f[0] == "dram__bytes_read.sum":
+                rd = float(f[1]) * unit.get(f[2], 1.0)
+            if len(f) >= 3 and f[0] == "dram__bytes_write.sum":
+                wr = float(f[1]) * unit.get(f[2], 1.0)
+    if rd is None or wr is None:
+        return None, "kernel not found in " + os.path.relpath(path, ROOT)
+    return rd + wr, os.path.relpath(path, ROOT) + " (ncu, committed capture of this workload)"
+
+
 def aggregate_replicas(total_ms, e2e_s, rows, world, device):
     """Whole-job numbers of `world` independent replicas: the slowest rank's times, the sum of the rows."""
     if world <= 1:
@@ -127,12 +158,12 @@ def aggregate_replicas(total_ms, e2e_s, rows, world, device):
     return float(tmax[0]), float(tmax[1]), float(tsum[2])
 
 
-def build_pair(wl, device):
+def build_pair(wl, device, rollout_layers=0):
     from paper_2509_23094_b200 import binding
     w_cpu = inputs.make_weights(wl.shape, seed=wl.seed, device=device if wl.shape.n_layers > 4 else "cpu")
     w_dev = {"layers": [{k: (None if v is None else v.to(device)) for k, v in lyr.items()} for lyr in w_cpu["layers"]],
              "g_final": w_cpu["g_final"].to(device), "w_lm": w_cpu["w_lm"].to(device), "embed": w_cpu["embed"].to(device)}
-    cfg = binding.make_config(wl.shape, wl.batch, wl.seq_len, sigma=wl.sigma)
+    cfg = binding.make_config(wl.shape, wl.batch, wl.seq_len, sigma=wl.sigma, rollout_layers=rollout_layers)
     ctx = binding.Context(cfg, w_dev, device=device)
     mask = inputs.make_mask(wl)
     tokens = inputs.make_tokens(wl, mask)
@@ -146,7 +177,7 @@ def run_ours(args, rank, world, device):
         from dataclasses import replace as _replace
         wl = _replace(wl, p=wl.p if args.p is None else args.p, k=wl.k if args.k is None else args.k)
     shape, B, L, d = wl.shape, wl.batch, wl.seq_len, wl.shape.d_model
-    w_cpu, w_dev, ctx, mask, tokens, h0 = build_pair(wl, device)
+    w_cpu, w_dev, ctx, mask, tokens, h0 = build_pair(wl, device, args.rollout_layers)
     mask_dev = mask.to(device)
     stream = torch.cuda.current_stream()
 
@@ -167,8 +198,6 @@ def run_ours(args, rank, world, device):
             ctx.view(n, B, L).copy_(t)
         flush.fill_(1)
 
-    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     sampler = ClockSampler(torch.cuda.current_device())
     for _ in range(args.warmup):
         restore()
@@ -180,19 +209,22 @@ def run_ours(args, rank, world, device):
     n_b = [int(row_off[b + 1] - row_off[b]) for b in range(B)]
     n, n_m = int(row_off[B]), int(lm_off[B])
 
-    def timed_pass(profile):
-        """K steps, each bracketed by CUDA events on the step's stream; state restored and L2 flushed between steps."""
+    def timed_pass(profile, steps, p=None):
+        """`steps` steps, each bracketed by CUDA events on the step's stream; state restored and L2 flushed between steps."""
+        p = wl.p if p is None else p
+        e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
         if profile:
             ctx.profile(True)
             ctx.profile_read(reset=True)
-        for i in range(args.steps):
+        for i in range(steps):
             restore()
-            ev0[i].record(stream)
-            ctx.step(h0, mask_dev, wl.k, wl.p, hidden_out=hid)
-            ev1[i].record(stream)
+            e0[i].record(stream)
+            ctx.step(h0, mask_dev, wl.k, p, hidden_out=hid)
+            e1[i].record(stream)
         torch.cuda.synchronize()
         if world > 1:
             torch.distributed.barrier()
@@ -200,17 +232,22 @@ def run_ours(args, rank, world, device):
         if profile:
             ph = ctx.profile_read(reset=True)
             ctx.profile(False)
-        return [a.elapsed_time(b) for a, b in zip(ev0, ev1)], ph
+        return [a.elapsed_time(b) for a, b in zip(e0, e1)], ph
 
-    # Pass 1 gives the headline: no events inside the step, so the kernels' programmatic dependent
-    # launches overlap as they do for a user.  Pass 2 repeats the same K steps with one event at every
-    # phase boundary (which serialises the launches) and gives the per-phase and per-kernel times.
+    # Pass 1 gives the headline: exactly K steps with no events inside the step, so the kernels' programmatic
+    # dependent launches overlap as they do for a user.  Pass 2 repeats the step with one event at every phase
+    # boundary (which serialises the launches) and gives the per-phase and per-kernel times; it runs long enough
+    # (at least 100 steps of the short workloads) for the clock sampler to collect a usable number of readings.
+    prof_steps = args.steps if shape.n_layers > 4 else max(args.steps, 100)
     sampler.start()
-    per_step_ms, _ = timed_pass(False)
-    per_step_ms_profiled, phases = timed_pass(True)
+    per_step_ms, _ = timed_pass(False, args.steps)
+    per_step_ms_profiled, phases = timed_pass(True, prof_steps)
     clocks = sampler.stop()
     ctx.sync_status()
     total_ms = sum(per_step_ms)
+    # SM clock inside the last profiled gate/up launch: clock64 against the global timer, stamped by CTA 0
+    gc = ctx.view("gemm_clocks").cpu().tolist()
+    mhz_in_gemm = round((gc[2] - gc[0]) / (gc[3] - gc[1]) * 1e3, 1) if gc[3] > gc[1] else None
 
     # end to end: host buffers in, host results out, through d2c_step_host
     h0_host = h0.cpu().pin_memory(); mask_host = mask.pin_memory()
@@ -235,36 +272,50 @@ def run_ours(args, rank, world, device):
     e2e_value = n_all / (e2e_s / e2e_steps)
 
     peaks = measured_peaks()
-    depth = shape.n_layers
+    depth = args.rollout_layers if 0 < args.rollout_layers < shape.n_layers else shape.n_layers
     flops, byts = algorithmic_work(shape, B, L, n_b, n_m, depth)
     t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
-    # dominant kernel: the gate/up projection GEMM (gemm_tc2_kernel<EPI_SWIGLU>, one launch per layer); its
-    # average launch duration comes from the events of the second timed pass
-    gu_ms = phases["gemm_gate_up"]["ms"] / args.steps / shape.n_layers
-    gu_flops = 2 * n * d * 2 * shape.d_ffn
-    achieved = gu_flops / (gu_ms * 1e-3) / 1e12 if gu_ms > 0 else 0.0
-    gemm_ms = sum(phases[k]["ms"] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) / args.steps
-    gemm_flops = shape.n_layers * 2 * n * shape.params_per_layer
     # Denominator: the burst cuBLAS figure for a kernel inside a short step; the sustained one when the clock
     # record of the timed region shows the power cap holding the SM clock below 90 % of its maximum.
     capped = "sw_power_cap" in clocks.get("reasons", []) and clocks.get("sm_mhz", 0) < 0.9 * (clocks.get("sm_max_mhz") or 0)
     tensor_peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
     peak_kind = " sustained (power-capped step)" if capped else " burst"
-    # DRAM bytes of one launch from the committed ncu capture of this workload (profiles/), null elsewhere
-    traffic = 229.7e6 if wl.name == "llada1l_1024" else None
-    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel<SWIGLU> (gate/up projection, 1 launch per layer)",
+    # Per-kernel figures come from the events of the second (profiled) pass.  The four projection GEMMs of a
+    # layer are tensor-bound at this row count, the LM head streams its weights once and is HBM-bound.
+    Hq, Hkv, Dh, F = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn
+    gemm_shapes = {"gemm_qkv": (d, (Hq + 2 * Hkv) * Dh), "gemm_o": (Hq * Dh, d), "gemm_gate_up": (d, 2 * F), "gemm_down": (F, d)}
+    gemms = {}
+    for name, (kk, nn) in gemm_shapes.items():
+        ms = phases[name]["ms"] / prof_steps / shape.n_layers
+        tf = 2.0 * n * kk * nn / (ms * 1e-3) / 1e12 if ms > 0 else 0.0
+        gemms[name] = {"launch_ms": round(ms, 4), "achieved": round(tf, 1), "frac": round(tf / tensor_peak, 4)}
+    gu_ms = gemms["gemm_gate_up"]["launch_ms"]
+    achieved = gemms["gemm_gate_up"]["achieved"]
+    gemm_ms = sum(phases[k]["ms"] for k in gemm_shapes) / prof_steps
+    gemm_flops = shape.n_layers * 2 * n * shape.params_per_layer
+    # DRAM bytes of one gate/up launch: read from the committed ncu summary of this workload, null elsewhere
+    traffic, traffic_source = (profiled_traffic("gate/up") if wl.name == "llada1l_1024" and args.p is None and args.scores == "rollout"
+                               else (None, "no capture of this workload"))
+    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel<SWIGLU> (gate/up projection, 1 launch per layer; the GEMM with the most FLOPs)",
                 "achieved": round(achieved, 2), "peak": tensor_peak, "peak_source": peaks["source"] + peak_kind,
                 "unit": "TFLOP/s", "frac": round(achieved / tensor_peak, 4),
-                "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4), "traffic": traffic,
+                "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4), "traffic": traffic, "traffic_source": traffic_source,
                 "algorithmic_bytes": 2 * d * 2 * shape.d_ffn + n * d * 2 + n * shape.d_ffn * 2,
                 "launch_ms": round(gu_ms, 4),
+                # what the launch took in SM clocks: by the NVML samples of the timed region, and by the clock the
+                # kernel itself saw (clock64 against the global timer inside CTA 0)
+                "launch_cycles_at_sampled_clock": round(gu_ms * 1e-3 * (clocks.get("sm_mhz") or 0) * 1e6),
+                "sm_mhz_inside_launch": mhz_in_gemm,
+                "launch_cycles_at_kernel_clock": round(gu_ms * 1e-3 * mhz_in_gemm * 1e6) if mhz_in_gemm else None,
+                "gemms": gemms,
                 "all_gemms": {"achieved": round(gemm_flops / (gemm_ms * 1e-3) / 1e12, 2) if gemm_ms > 0 else 0.0,
                               "ms_per_step": round(gemm_ms, 4)},
                 "step_roofline_ms": round(t_roof * 1e3, 4), "step_frac": round(t_roof * 1e3 / ms_per_step, 4),
                 "step_flops": flops, "step_bytes": byts}
-    lm_ms = phases["lm_head"]["ms"] / args.steps
+    lm_ms = phases["lm_head"]["ms"] / prof_steps
     lm_bytes = 2 * d * shape.vocab
-    roofline["lm_head"] = {"bound": "hbm", "achieved": round(lm_bytes / (lm_ms * 1e-3) / 1e9, 1) if lm_ms > 0 else 0.0,
+    roofline["lm_head"] = {"bound": "hbm", "kernel": "gemm_tc_kernel<LMSTATS> (the longest single launch of the step)",
+                           "achieved": round(lm_bytes / (lm_ms * 1e-3) / 1e9, 1) if lm_ms > 0 else 0.0,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": round(lm_bytes / (lm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4) if lm_ms > 0 else 0.0,
                            "ms_per_step": round(lm_ms, 4)}
@@ -275,16 +326,42 @@ def run_ours(args, rank, world, device):
         "config": {"workload": wl.name, "shape": shape.name, "batch": B, "seq_len": L, "k": wl.k, "p": wl.p,
                    "selected_rows": n_b, "lm_rows": n_m, "l2": "flushed between steps; weights (%.2f GB) exceed L2" %
                    ((2 * shape.n_layers * shape.params_per_layer + 2 * d * shape.vocab) / 1e9),
-                   "replicas": world, "scores": args.scores},
+                   "replicas": world, "scores": args.scores, "rollout_layers": depth},
         "clocks": clocks,
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": round(e2e_s / e2e_steps * 1e3, 4)},
-        "gpu_launches": int(sum(p["launches"] for p in phases.values())),
+        "gpu_launches": int(round(sum(p["launches"] for p in phases.values()) * args.steps / prof_steps)),
         "roofline": roofline,
-        "phases_ms_per_step": {k: round(v["ms"] / args.steps, 4) for k, v in phases.items()},
+        "phases_ms_per_step": {k: round(v["ms"] / prof_steps, 4) for k, v in phases.items()},
         "step_ms_min": round(min(per_step_ms), 4), "step_ms_median": round(statistics.median(per_step_ms), 4),
-        "ms_per_step_with_phase_events": round(sum(per_step_ms_profiled) / args.steps, 4),
+        "ms_per_step_with_phase_events": round(sum(per_step_ms_profiled) / prof_steps, 4), "profiled_steps": prof_steps,
     }
+    # The same workload at the paper's default threshold (Section 5.1: p = 0.1, about a hundred selected rows:
+    # the weight-streaming regime), as a labelled extra; the library picks its few-row kernels from the previous
+    # step's row count, so two untimed steps come first.
+    if rank == 0 and world == 1 and shape.n_layers <= 4 and args.p is None and args.scores == "rollout" and not args.no_extras:
+        for _ in range(3):
+            restore()
+            ctx.step(h0, mask_dev, wl.k, 0.1, hidden_out=hid)
+            torch.cuda.synchronize()
+        ro01 = ctx.view("row_off", B, L).cpu().numpy(); lo01 = ctx.view("lm_off", B, L).cpu().numpy()
+        nb01 = [int(ro01[b + 1] - ro01[b]) for b in range(B)]
+        ms01, _ = timed_pass(False, args.steps, p=0.1)
+        _, ph01 = timed_pass(True, prof_steps, p=0.1)
+        fl01, by01 = algorithmic_work(shape, B, L, nb01, int(lo01[B]), depth)
+        roof01 = max(fl01 / (peaks["bf16_tflops"] * 1e12), by01 / (peaks["hbm_gbs"] * 1e9))
+        g01 = sum(ph01[k]["ms"] for k in gemm_shapes) / prof_steps
+        wbytes = 2 * shape.n_layers * shape.params_per_layer
+        line["paper_default_p0.1"] = {
+            "selected_rows": nb01, "lm_rows": int(lo01[B]), "ms_per_step": round(sum(ms01) / args.steps, 4),
+            "step_roofline_ms": round(roof01 * 1e3, 4), "step_frac": round(roof01 * 1e3 / (sum(ms01) / args.steps), 4),
+            "all_gemms": {"ms_per_step": round(g01, 4), "weight_gbs": round(wbytes / (g01 * 1e-3) / 1e9, 1) if g01 > 0 else 0.0,
+                          "frac_of_hbm": round(wbytes / (g01 * 1e-3) / 1e9 / peaks["hbm_gbs"], 4) if g01 > 0 else 0.0},
+            "phases_ms_per_step": {k: round(v["ms"] / prof_steps, 4) for k, v in ph01.items()}}
+        for _ in range(2):                                    # back to the workload's own regime
+            restore()
+            ctx.step(h0, mask_dev, wl.k, wl.p, hidden_out=hid)
+            torch.cuda.synchronize()
     if args.decode:
         line["decode"] = decode_loop(ctx, wl, w_dev, mask, tokens, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -368,7 +445,7 @@ def cpu_baseline(wl, w_cpu, mask, tokens, ctx, B, L, max_rows=1024):
         ostep.oracle_step(st, wf, wl.shape, h0, mask.numpy(), k=0, p=0.0, sigma=wl.sigma, sel_override=sample)
         dt += time.perf_counter() - t0
         reps += 1
-    return {"value": round(rows * reps / dt, 2), "unit": UNIT, "kind": "oracle", "cores": blas_threads(),
+    return {"value": round(rows * reps / dt, 2), "unit": UNIT, "kind": "oracle (fp64 numpy, as it stands)", "cores": blas_threads(),
             "sample": f"{reps} oracle steps, each on {rows} of the selected rows (fp64 numpy), {dt:.1f} s in all"}
 
 
@@ -412,7 +489,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 2), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "shape": wl.shape.name, "batch": B, "seq_len": L, "k": wl.k, "p": wl.p},
-        "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "kind": "oracle", "cores": blas_threads(), "sample": desc},
+        "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "kind": "oracle (fp64 numpy, as it stands)", "cores": blas_threads(), "sample": desc},
         "e2e": {"value": round(value, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
@@ -427,10 +504,22 @@ def main():
     ap.add_argument("--decode", action="store_true", help="also run the workload's whole decoding loop")
     ap.add_argument("--p", type=float, default=None, help="override the workload's top-p threshold (e.g. the paper's default 0.1)")
     ap.add_argument("--k", type=int, default=None, help="override the workload's k")
+    ap.add_argument("--rollout-layers", type=int, default=0,
+                    help="roll the attention out over the first n layers only (the paper's Rollout-5 variant); 0 = all layers")
+    ap.add_argument("--no-extras", action="store_true", help="skip the labelled extra run at the paper's default p = 0.1")
     ap.add_argument("--scores", default="rollout", choices=["rollout", "zipf"],
                     help="stage-2 scores before each timed step: the prefill's rollout (default) or a seeded Zipf(1.0)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: start the N ranks ourselves (one process per GPU, rendezvous on the loopback address)
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -176,6 +176,9 @@ typedef struct {
   float*   abar;        /* f32 [n_layers][max_batch*max_seq][max_seq] head-averaged attention rows   */
   float*   lse;         /* f32 [max_batch*max_seq][Hq] log-sum-exp of the last layer's scores        */
   int32_t* status;      /* [4] device status word: [0] error code, [1] where                         */
+  int64_t* gemm_clocks; /* [4] while d2c_profile is on: SM clock counter and global timer (ns) at the start
+                           and at the end of CTA 0 of the last gate/up projection launch, i.e. the SM
+                           clock that launch really ran at: ([2]-[0]) / ([3]-[1]) GHz                 */
 } d2c_state;
 /* The per-position vectors (conf, pred, c, key) are indexed [b*seq_len + pos] with the batch and
  * seq_len of the d2c_step calls; a context is used with one (batch, seq_len) from its first step on

@@ -60,7 +60,7 @@ class HostOut(C.Structure):
 
 class State(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("kcache", "vcache", "conf", "pred", "c", "key", "sel_idx", "row_off",
-                                          "lm_rows", "lm_off", "abar", "lse", "status")]
+                                          "lm_rows", "lm_off", "abar", "lse", "status", "gemm_clocks")]
 
 
 _lib = None
@@ -204,6 +204,8 @@ class Context:
             return self._view(self.state.lse, R * c.n_q_heads, torch.float32).view(R, c.n_q_heads)
         if name == "status":
             return self._view(self.state.status, 4, torch.int32)
+        if name == "gemm_clocks":
+            return self._view(self.state.gemm_clocks, 4, torch.int64)
         raise KeyError(name)
 
     def abar(self, layer: int, n_rows: int, seq_len: int) -> torch.Tensor:

@@ -32,6 +32,7 @@ void count_launch(int n);
 // attribute and starts with pdl_prologue(), which waits for the preceding kernel's results and then
 // lets the following kernel begin its own launch, so launch latency overlaps the predecessor's tail.
 #ifdef __CUDACC__
+__device__ __forceinline__ long long global_timer_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 __device__ __forceinline__ void pdl_prologue() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -119,6 +120,9 @@ struct GemmArgs {
   // split-K scratch of the one-SM tcgen05 kernel (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
   // and as many zero-initialised arrival counters
   float* sk_partials; int32_t* sk_counters; int sk_max_tiles;
+  // optional (tcgen05 kernels): CTA 0 stores {clock64, globaltimer ns} at its start and its end, which gives the
+  // SM clock the launch really ran at (a power-capped clock is not what a coarse NVML sample shows)
+  long long* clock_probe;
 };
 static const int kSkMaxTiles = 160;
 int launch_gemm_mma(const GemmArgs& g, GemmEpilogue epi, cudaStream_t st);

@@ -54,7 +54,7 @@ struct Buffers {
   bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar;
   float *st_max, *st_sum; int32_t* st_arg;
   float *u0, *u1, *partial;
-  float* sk_partials; int32_t* sk_counters;
+  float* sk_partials; int32_t* sk_counters; long long* gemm_clocks;
   float* abar_part; size_t abar_part_floats;
   bf16* h0_stage; uint8_t* mask_stage; int32_t *forced_stage, *forced_off_stage; float *okey_stage, *oc_stage;
   int32_t* committed_stage;
@@ -87,6 +87,7 @@ static size_t carve(const d2c_config& c, void* base, Buffers* out) {
   b.u0 = w.take<float>(R); b.u1 = w.take<float>(R);
   b.partial = w.take<float>((size_t)kRolloutSplit * R + (R + 3) / 4);     // partial sums + selected-flag bytes
   b.sk_partials = w.take<float>((size_t)kSkMaxTiles * 128 * 256); b.sk_counters = w.take<int32_t>(kSkMaxTiles);
+  b.gemm_clocks = w.take<long long>(4);
   // scratch for the head-split of the abar kernel: only worth having when the (rows x keys) grid is small
   const size_t tiles_worst = (size_t)ceil_div((int)L, 128) * ceil_div((int)L, 128) * B;
   b.abar_part_floats = tiles_worst < 2 * 160 ? (size_t)8 * R * L : 0;
@@ -322,7 +323,7 @@ int d2c_state_ptrs(d2c_ctx* ctx, d2c_state* out) {
   const Buffers& b = ctx->buf;
   out->kcache = b.kcache; out->vcache = b.vcache; out->conf = b.conf; out->pred = b.pred; out->c = b.c; out->key = b.key;
   out->sel_idx = b.sel_idx; out->row_off = b.row_off; out->lm_rows = b.lm_rows; out->lm_off = b.lm_off;
-  out->abar = b.abar; out->lse = b.lse; out->status = b.status;
+  out->abar = b.abar; out->lse = b.lse; out->status = b.status; out->gemm_clocks = reinterpret_cast<int64_t*>(b.gemm_clocks);
   return D2C_OK;
 }
 
@@ -492,6 +493,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     GemmArgs gf{};
     gf.A = b.xn; gf.lda = d; gf.W = ctx->w_gate[l]; gf.W2 = ctx->w_up[l]; gf.C = b.hmid; gf.ldc = c.d_ffn;
     gf.n_rows = n_rows; gf.max_rows = R; gf.N = c.d_ffn; gf.K = d;
+    gf.clock_probe = ctx->prof ? b.gemm_clocks : nullptr;
     D2C_TRY(ctx, gemm(ctx, gf, EPI_SWIGLU));
     GemmArgs gd{};
     gd.A = b.hmid; gd.lda = c.d_ffn; gd.W = ctx->w_down[l]; gd.C = x; gd.ldc = d; gd.n_rows = n_rows; gd.max_rows = R; gd.N = d; gd.K = c.d_ffn;

@@ -92,6 +92,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   volatile int* abortp = &abort_flag;
 
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
   const int n = max(*g.n_rows, 0);
   const int MT = (n + TM - 1) / TM;
   const int KT = g.K / TK, G = gridDim.x;
@@ -356,6 +357,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     tc_fence_after();
     tmem_dealloc(tmem_acc, 2 * ACC_COLS);
   }
+  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[2] = clock64(); g.clock_probe[3] = global_timer_ns(); }
 }
 
 template <int EPI>

@@ -117,6 +117,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   volatile int* abortp = &abort_flag;
 
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
   const int n = *g.n_rows;
   const int MT = (max(n, 0) + 2 * TM - 1) / (2 * TM);
   const int KT = g.K / TK;
@@ -357,6 +358,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after();
     tmem_dealloc2(tmem_acc, 2 * ACC_COLS);
   }
+  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[2] = clock64(); g.clock_probe[3] = global_timer_ns(); }
 }
 
 template <int EPI>
