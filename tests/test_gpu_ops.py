@@ -33,6 +33,21 @@ def test_gemm_matches_fp64(impl, rows, n, N, K):
         assert np.all(got[n:] == 0)                                   # rows past n_rows are not written
 
 
+@pytest.mark.parametrize("n", [769, 835, 896, 897, 1023, 1024, 40, 128, 129])
+def test_gemm_ragged_row_counts_on_the_pair_kernel(n):
+    """Row counts around the 256-row pair tile (one row, 67, 128, 129 and 255 rows in the last tile, and fewer
+    rows than one CTA holds) with enough column tiles that the launch keeps full-width tiles and takes no split-K."""
+    rows, N, K = 1024, 4864, 128
+    A = _bf16((rows, K), 11); W = _bf16((N, K), 12, 0.05); bias = _bf16((N,), 13)
+    n_dev = torch.tensor([n], dtype=torch.int32, device="cuda")
+    Cm = binding.d2c_op_gemm(A.cuda(), W.cuda(), n_dev, bias=bias.cuda(), impl=0)
+    torch.cuda.synchronize()
+    want = A.double().numpy()[:n] @ W.double().numpy().T + bias.double().numpy()
+    got = Cm.float().cpu().numpy()
+    assert row_rel_err(got[:n], want) <= ROW_TOL / 4
+    assert np.all(got[n:] == 0)
+
+
 def _attention_ref(q, kc, vc, row_off, L, Hq, Hkv, Dh):
     rows = q.shape[0]
     o = np.zeros((rows, Hq * Dh)); lse = np.zeros((rows, Hq)); abar = np.zeros((rows, L))

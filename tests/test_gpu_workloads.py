@@ -63,7 +63,7 @@ class Runner:
             np.testing.assert_array_equal(S[b], want, err_msg=f"sequence {b}")
         return ro, S
 
-    def check_layers(self, ro, S, layers, rows_per_seq=64, seqs=None, seed=0):
+    def check_layers(self, ro, S, layers, rows_per_seq=64, seqs=None, seed=0, local_rows=None):
         wl, shape = self.wl, self.shape
         B, L, d = wl.batch, wl.seq_len, shape.d_model
         rng = np.random.default_rng(seed)
@@ -76,7 +76,7 @@ class Runner:
                 nb = len(S[b])
                 if nb == 0:
                     continue
-                pick = np.sort(rng.choice(nb, min(rows_per_seq, nb), replace=False))
+                pick = np.sort(rng.choice(nb, min(rows_per_seq, nb), replace=False)) if local_rows is None else np.asarray(local_rows)
                 rows = ro[b] + pick
                 pos = S[b][pick]
                 x_in = _f64(self.layer_in[l][rows])
@@ -175,6 +175,30 @@ def test_llada_single_layer_1024_few_rows():
     r.check_layers(ro, S, [0], seqs=[0])
     r.check_lm_head()
     r.check_rollout(ro, S, [0])
+    kc1 = r.ctx.view("kcache"); vc1 = r.ctx.view("vcache")
+    keep = torch.ones(L, dtype=torch.bool, device="cuda"); keep[torch.from_numpy(S[0]).cuda()] = False
+    assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
+
+
+@pytest.mark.parametrize("n_sel", [257, 323, 384, 385, 511, 835])
+def test_llada_single_layer_row_counts_around_the_pair_tile(n_sel):
+    """Selected-row counts with n mod 256 in {1, 67, 128, 129, 255}: the ragged last row tile of every projection
+    (fused QKV + rotary + cache scatter, residual, SwiGLU), all of its rows checked.  The rows are forced so
+    that the count is exact; k = 0 and p = 0 select nothing else."""
+    wl = inputs.WORKLOADS["llada1l_1024"]
+    r = Runner(wl)
+    B, L = wl.batch, wl.seq_len
+    r.step(10 ** 6, 1.0)
+    rng = np.random.default_rng(n_sel)
+    forced = [sorted(rng.choice(L, n_sel, replace=False).tolist())]
+    kc0 = r.ctx.view("kcache").clone(); vc0 = r.ctx.view("vcache").clone()
+    ro, S = r.step(0, 0.0, forced=forced)
+    assert len(S[0]) == n_sel
+    # every row of the last, ragged tile and a sample of the others
+    tail = np.arange((n_sel - 1) // 256 * 256, n_sel)
+    r.check_layers(ro, S, [0], rows_per_seq=48, seqs=[0], seed=n_sel)
+    r.check_layers(ro, S, [0], seqs=[0], local_rows=tail[:: max(1, len(tail) // 48)])
+    r.check_lm_head()
     kc1 = r.ctx.view("kcache"); vc1 = r.ctx.view("vcache")
     keep = torch.ones(L, dtype=torch.bool, device="cuda"); keep[torch.from_numpy(S[0]).cuda()] = False
     assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
