@@ -3,43 +3,27 @@
 // One CTA per sequence.  Every sum that decides an index is an integer sum, so the result does
 // not depend on the order in which threads add:
 //   stage 1 (Eq. 3-4): D(i) = sum over known j of phi(|i-j|), with phi tabulated as round(phi*2^30);
-//                      key = fp32(D) * conf (one multiply); the k largest keys among masked positions.
-//   stage 2 (after Eq. 9): candidates sorted by score c_j (ties: lower position first); the shortest
+//                      key = fp32(D) * conf (one multiply); the k largest keys among masked positions
+//                      (equal keys: lower position first).
+//   stage 2 (after Eq. 9): candidates in the order (score c_j descending, position ascending); the shortest
 //                      prefix whose mass sum floor(c_j*2^32) exceeds p times the total.
-// Sorting is a bitonic network over 64-bit words (score bits << 32 | ~position) in shared memory.
+// Neither stage sorts.  Both are "take elements in that order until a running weight crosses a threshold"
+// (weight 1 and threshold k for stage 1, the fixed-point mass and p * total for stage 2), which needs only the
+// score value at which the crossing happens: four 8-bit radix passes over the fp32 bit patterns, each a
+// 256-bin histogram of weights scanned from the top, find it exactly; elements above that value are taken,
+// elements equal to it are taken in position order while the running weight has not crossed.  Up to 1024
+// masked positions (every decoding step of the workloads) stage 1 skips even that and ranks each masked
+// position against all others directly, one position per thread.
 #include <math.h>
 
 #include "common.cuh"
 
 namespace d2c {
 
-static constexpr int kSelThreads = 1024;
+static constexpr int kSelThreads = 512;
 static constexpr int kPhiMax = 512;              // phi entries kept in shared memory; a wider window reads the rest from global memory
+static constexpr int kRankMax = 1024;            // stage 1 ranks by direct comparison up to this many masked positions
 enum : uint8_t { F_SEL = 1, F_MSTAR = 2 };
-
-// Descending bitonic sort of n 64-bit words in shared memory by the whole block.  Pair p of a stage exchanges
-// elements lo = 2p - (p & (stride - 1)) and lo + stride; for stride <= 32 the pairs of one warp touch only that
-// warp's 64 elements, so only the stages that reach further need the block to synchronise.  (Keeping the words in
-// registers and exchanging by warp shuffles was no faster: with 32 warps on one SM the stages are bound by
-// instruction issue, not by the shared-memory round trip.)
-__device__ __forceinline__ void bitonic_sort_desc(uint64_t* buf, int n) {
-  bool wide_before = true;                                  // the caller's writes count as a block-wide stage
-  for (int size = 2; size <= n; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      const bool wide = stride >= 64;
-      if (wide || wide_before) __syncthreads(); else __syncwarp();
-      wide_before = wide;
-      for (int t = threadIdx.x; t < (n >> 1); t += blockDim.x) {
-        const int lo = 2 * t - (t & (stride - 1));
-        const int hi = lo + stride;
-        const bool desc = (lo & size) == 0;
-        const uint64_t x = buf[lo], y = buf[hi];
-        if ((x < y) == desc) { buf[lo] = y; buf[hi] = x; }
-      }
-    }
-  }
-  __syncthreads();
-}
 
 // Exclusive block scan of one value per thread; returns the exclusive prefix, *total gets the sum.
 template <typename T>
@@ -74,201 +58,266 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* warp_buf, T* total) {
 // mass of 8192 positions stays inside 64 bits.
 __device__ __forceinline__ float clean_score(float x) { return (x > 0.f && x < INFINITY) ? fminf(x, 262144.f) : 0.f; }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a, int P2) {
+// Shared scratch of the threshold search.
+struct RadixScratch {
+  unsigned long long hist[256];            // per digit: the weight sum of the members that carry it
+  unsigned long long warp_buf[32];
+  unsigned long long total;
+  unsigned long long above;
+  int digit;                               // crossing digit of the pass, -1: the weight of all members does not cross
+};
+
+__device__ __forceinline__ unsigned long long shfl_up_u64(unsigned long long v, int o) {
+  const uint32_t lo = __shfl_up_sync(0xffffffffu, (uint32_t)v, o), hi = __shfl_up_sync(0xffffffffu, (uint32_t)(v >> 32), o);
+  return ((unsigned long long)hi << 32) | lo;
+}
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int o) {
+  const uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, o), hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(v >> 32), o);
+  return ((unsigned long long)hi << 32) | lo;
+}
+
+// The shortest prefix, in the order (value bits descending, position ascending), of the positions j < L with
+// member(j) whose running weight "crosses": crossed(w) must be monotone in w and false for w = 0.  Sets `mark`
+// in flags for every position of that prefix; if the weight never crosses, for every member.
+// weight(bits) is 1 (counting) or the fixed-point mass; all members with equal bits have equal weight.
+// rs.hist must be zero on entry and is zero again on return.
+// [vmin, vmax] bounds the members' value bits: leading digits on which the two agree need no pass.
+template <typename Member, typename Weight, typename Crossed>
+__device__ __forceinline__ void take_until_crossed(const uint32_t* vb, int L, Member member, Weight weight, Crossed crossed,
+                                                   uint8_t* flags, uint8_t mark, RadixScratch& rs, uint32_t vmin, uint32_t vmax) {
+  const int tid = threadIdx.x, lane = tid & 31, T = blockDim.x;
+  uint32_t pref = 0;                                     // the high digits fixed so far
+  unsigned long long above = 0;                          // weight of the members above the range still searched
+  bool all = false;
+  int pass0 = 0;
+  while (pass0 < 3 && (vmin >> (24 - 8 * pass0)) == (vmax >> (24 - 8 * pass0))) ++pass0;
+  if (pass0 > 0) pref = vmax >> (32 - 8 * pass0);
+  for (int pass = pass0; pass < 4 && !all; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int base = 0; base < L; base += T) {
+      const int j = base + tid;
+      const bool m = j < L && member(j) && (pass == 0 || (vb[j] >> (shift + 8)) == pref);
+      const unsigned act = __ballot_sync(0xffffffffu, m);
+      if (act) {
+        // a warp whose live lanes all carry the same digit (flat scores, the high digits) adds once; otherwise each lane adds
+        const uint32_t d = m ? (vb[j] >> shift) & 255u : 0u;
+        unsigned long long w = m ? weight(vb[j]) : 0ull;
+        const int leader = __ffs(act) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, d, leader);
+        if (__all_sync(0xffffffffu, !m || d == d0)) {
+          for (int o = 16; o > 0; o >>= 1) w += shfl_xor_u64(w, o);
+          if (lane == leader && w) atomicAdd(&rs.hist[d0], w);
+        } else if (m && w) {
+          atomicAdd(&rs.hist[d], w);
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // one warp walks the digits from the top: lane l owns digits 255 - 8 l down to 248 - 8 l
+      unsigned long long w[8], sum = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int bin = 255 - (8 * lane + k);
+        w[k] = rs.hist[bin];
+        rs.hist[bin] = 0;
+        sum += w[k];
+      }
+      unsigned long long inc = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = shfl_up_u64(inc, o);
+        if (lane >= o) inc += up;
+      }
+      unsigned long long run = above + inc - sum;        // weight above this lane's first digit
+      int hit = -1; unsigned long long before = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (hit < 0 && w[k] != 0 && crossed(run + w[k])) { hit = k; before = run; }
+        run += w[k];
+      }
+      const unsigned found = __ballot_sync(0xffffffffu, hit >= 0);
+      if (found == 0) {
+        if (lane == 0) rs.digit = -1;
+      } else if (lane == __ffs(found) - 1) {
+        rs.digit = 255 - (8 * lane + hit);
+        rs.above = before;
+      }
+    }
+    __syncthreads();
+    if (rs.digit < 0) {
+      all = true;                                        // the weight of all members together does not cross
+    } else {
+      above = rs.above;
+      pref = (pref << 8) | (uint32_t)rs.digit;
+    }
+    // (rs.digit is rewritten only behind the next pass's barrier)
+  }
+  // members above the crossing value are in; those equal to it, in position order, while the weight before them has not crossed
+  const int per = (L + T - 1) / T;
+  const int j0 = tid * per;
+  unsigned long long ties = 0;
+  if (!all)
+    for (int e = 0; e < per; ++e) {
+      const int j = j0 + e;
+      if (j < L && member(j) && vb[j] == pref) ++ties;
+    }
+  unsigned long long r = all ? 0ull : block_exclusive_scan<unsigned long long>(ties, rs.warp_buf, &rs.total);
+  const unsigned long long wstar = weight(pref);
+  for (int e = 0; e < per; ++e) {
+    const int j = j0 + e;
+    if (j >= L || !member(j)) continue;
+    bool in = all || vb[j] > pref;
+    if (!all && vb[j] == pref) { in = !crossed(above + r * wstar); ++r; }
+    if (in) flags[j] |= mark;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
   pdl_prologue();
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint64_t* sbuf = reinterpret_cast<uint64_t*>(smem_raw);
-  uint8_t* flags = reinterpret_cast<uint8_t*>(sbuf + P2);
-  uint8_t* smask = flags + a.seq_len;
-  __shared__ uint64_t warp_buf64[32];
-  __shared__ uint64_t s_total64;
+  const int b = blockIdx.x, L = a.seq_len, tid = threadIdx.x, lane = tid & 31;
+  uint32_t* kb = reinterpret_cast<uint32_t*>(smem_raw);       // stage-1 key bits (0 outside the stage-1 set)
+  uint32_t* cb = kb + L;                                       // stage-2 score bits
+  uint8_t* flags = reinterpret_cast<uint8_t*>(cb + L);
+  uint8_t* smask = flags + L;
+  uint8_t* in1 = smask + L;                                    // 1: masked and inside the block (the set stage 1 ranks)
+  __shared__ RadixScratch rsc;
+  __shared__ unsigned long long mlist[kRankMax];               // stage-1 members: position, then (key bits << 32 | ~position)
   __shared__ int warp_buf32[32];
-  __shared__ int s_total32, s_cnt, s_take;
+  __shared__ int s_total32, s_nm;
+  __shared__ unsigned long long s_mass;
+  __shared__ uint32_t s_lo, s_hi;
   __shared__ uint32_t s_phi[kPhiMax];                          // the non-zero head of the phi table (window +-65 at sigma 10)
 
-  const int b = blockIdx.x, L = a.seq_len, tid = threadIdx.x;
   const uint8_t* mask = a.mask + (size_t)b * L;
   const float* conf = a.conf + (size_t)b * L;
   const float* cs = a.c + (size_t)b * L;
   const float* okey = a.override_key ? a.override_key + (size_t)b * L : nullptr;
+  float* key_out = a.key + (size_t)b * L;
 
   // stage 1 may be confined to one block of positions (semi-autoregressive decoding); whole sequence otherwise
   const int blk_lo = a.block_hi > a.block_lo ? a.block_lo : 0, blk_hi = a.block_hi > a.block_lo ? a.block_hi : L;
-  for (int i = tid; i < L; i += kSelThreads) { smask[i] = mask[i] ? 1 : 0; flags[i] = 0; }
+  for (int i = tid; i < L; i += kSelThreads) {
+    smask[i] = mask[i] ? 1 : 0; flags[i] = 0; kb[i] = 0;
+    cb[i] = __float_as_uint(clean_score(cs[i]));
+  }
   for (int r = tid; r < min(a.phi_len, kPhiMax); r += kSelThreads) s_phi[r] = a.phi_q30[r];
-  if (tid == 0) { s_cnt = 0; }
+  for (int i = tid; i < 256; i += kSelThreads) rsc.hist[i] = 0;
+  if (tid == 0) { s_nm = 0; s_mass = 0; s_lo = 0xFFFFFFFFu; s_hi = 0u; }
   __syncthreads();
 
-  if (a.stage2_candidates == 0) {
-    // ---- default candidate mode: masked positions (stage 1) and known positions (stage 2) are disjoint,
-    //      so one sort orders both: bit 63 = masked, bits 62..32 = score bits, bits 31..0 = ~position ----
-    for (int i = tid; i < P2; i += kSelThreads) {
-      uint64_t comp = 0;
-      if (i < L) {
-        float key = 0.f;
-        if (smask[i] && i >= blk_lo && i < blk_hi) {
-          if (okey) {
-            key = clean_score(okey[i]);
-          } else {
-            unsigned long long dq = 0;
-            for (int r = 1; r < a.phi_len; ++r) {
-              const int lo = i - r, hi = i + r;
-              int known = 0;
-              if (lo >= 0) known += 1 - smask[lo];
-              if (hi < L) known += 1 - smask[hi];
-              dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * (unsigned)known;
-            }
-            const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;   // * 2^-30, exact
-            key = clean_score(__fmul_rn(D, conf[i]));
-          }
-          comp = (1ull << 63) | ((uint64_t)__float_as_uint(key) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
-        } else if (!smask[i]) {
-          comp = ((uint64_t)__float_as_uint(clean_score(cs[i])) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
-        }                                                           // masked outside the block: in neither stage
-        a.key[(size_t)b * L + i] = key;
-      }
-      sbuf[i] = comp;
+  // ---- the set stage 1 ranks: masked positions inside the block, listed in any order ----
+  for (int base = 0; base < L; base += kSelThreads) {
+    const int i = base + tid;
+    const bool m1 = i < L && smask[i] && i >= blk_lo && i < blk_hi;
+    if (i < L) { in1[i] = m1 ? 1 : 0; if (!m1) key_out[i] = 0.f; }
+    const unsigned act = __ballot_sync(0xffffffffu, m1);
+    if (act) {
+      int slot0 = 0;
+      if (lane == __ffs(act) - 1) slot0 = atomicAdd(&s_nm, __popc(act));
+      slot0 = __shfl_sync(0xffffffffu, slot0, __ffs(act) - 1);
+      const int slot = slot0 + __popc(act & ((1u << lane) - 1u));
+      if (m1 && slot < kRankMax) mlist[slot] = (unsigned long long)i;
     }
-    bitonic_sort_desc(sbuf, P2);
-    if (tid == 0) { s_cnt = 0; s_take = 0; }                      // s_take doubles as the masked count here
-    __syncthreads();
-    for (int t = tid; t < P2; t += kSelThreads) {
-      const uint64_t x = sbuf[t], y = t + 1 < P2 ? sbuf[t + 1] : 0ull;
-      if ((x >> 63) && !(y >> 63)) s_take = t + 1;
-      if (x != 0 && y == 0) s_cnt = t + 1;
+  }
+  __syncthreads();
+  const int nm = s_nm;
+
+  // ---- keys (Eq. 3-4): D(i) as an exact integer sum over the window, key = fp32(D) * confidence ----
+  auto known_at = [&](int i, int r) {
+    const int lo = i - r, hi = i + r;
+    int known = 0;
+    if (lo >= 0) known += 1 - smask[lo];
+    if (hi < L) known += 1 - smask[hi];
+    return (unsigned)known;
+  };
+  auto finish_key = [&](int i, unsigned long long dq, float cf) {
+    float key;
+    if (okey) {
+      key = clean_score(okey[i]);
+    } else {
+      const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;       // * 2^-30, exact
+      key = clean_score(__fmul_rn(D, cf));
     }
-    __syncthreads();
-    const int nm = s_take, ntot = s_cnt;
-    {
-      const int take = min(max(a.k, 0), nm);
-      for (int t = tid; t < take; t += kSelThreads) {
-        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
-        flags[idx] = F_SEL | F_MSTAR;
-      }
-    }
-    const int per = max(1, P2 / kSelThreads);
-    const int t0 = tid * per;
-    unsigned long long local = 0;
-    if (t0 < P2) {
-      for (int e = 0; e < per; ++e) {
-        const uint64_t x = sbuf[t0 + e];
-        if (!(x >> 63)) local += __double2ull_rd((double)__uint_as_float((uint32_t)(x >> 32)) * 4294967296.0);
-      }
-    }
-    const unsigned long long excl =
-        block_exclusive_scan<unsigned long long>(local, (unsigned long long*)warp_buf64, (unsigned long long*)&s_total64);
-    if (tid == 0) s_take = (a.p > 0.f) ? ntot : nm;                // end (exclusive) of the selected candidates
-    __syncthreads();
-    if (a.p > 0.f && t0 < P2) {
-      const double thr = __dmul_rn((double)a.p, __ull2double_rn(s_total64));
-      unsigned long long run = excl;
-      for (int e = 0; e < per; ++e) {
-        const int t = t0 + e;
-        if (t >= ntot) break;
-        if (t < nm) continue;
-        run += __double2ull_rd((double)__uint_as_float((uint32_t)(sbuf[t] >> 32)) * 4294967296.0);
-        if (__ull2double_rn(run) > thr) { atomicMin(&s_take, t + 1); break; }
+    key_out[i] = key;
+    kb[i] = __float_as_uint(key);
+    return key;
+  };
+  if (nm <= kRankMax) {
+    // a group of tpm lanes (a power of two, inside one warp) shares the window of one listed position
+    int tpm = 1;
+    while (tpm < 32 && 2 * tpm * nm <= kSelThreads) tpm <<= 1;
+    const int sub = tid & (tpm - 1), groups = kSelThreads / tpm;
+    for (int e0 = 0; e0 < nm; e0 += groups) {
+      const int e = e0 + tid / tpm;
+      const bool live = e < nm;
+      const int i = live ? (int)mlist[e] : 0;
+      const float cf = (live && sub == 0 && !okey) ? conf[i] : 0.f;       // in flight while the window is summed
+      unsigned long long dq = 0;
+      if (live && !okey)
+        for (int r = 1 + sub; r < a.phi_len; r += tpm)
+          dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * known_at(i, r);
+      for (int o = 1; o < tpm; o <<= 1) dq += shfl_xor_u64(dq, o);
+      __syncwarp();
+      if (live && sub == 0) {
+        const float key = finish_key(i, dq, cf);
+        mlist[e] = ((unsigned long long)__float_as_uint(key) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
       }
     }
-    __syncthreads();
-    {
-      const int end = s_take;
-      for (int t = nm + tid; t < end; t += kSelThreads) {
-        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
-        flags[idx] |= F_SEL;
-      }
-    }
-    __syncthreads();
   } else {
-  // ---- stage 1: keys ----
-  for (int i = tid; i < P2; i += kSelThreads) {
-    uint64_t comp = 0;
-    if (i < L) {
-      float key = 0.f;
-      if (smask[i] && i >= blk_lo && i < blk_hi) {
-        if (okey) {
-          key = clean_score(okey[i]);
-        } else {
-          unsigned long long dq = 0;
-          for (int r = 1; r < a.phi_len; ++r) {
-            const int lo = i - r, hi = i + r;
-            int known = 0;
-            if (lo >= 0) known += 1 - smask[lo];
-            if (hi < L) known += 1 - smask[hi];
-            dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * (unsigned)known;
-          }
-          const float D = __ull2float_rn(dq) * 9.31322574615478515625e-10f;   // * 2^-30, exact
-          key = clean_score(__fmul_rn(D, conf[i]));
-        }
-        comp = ((uint64_t)__float_as_uint(key) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
-      }
-      a.key[(size_t)b * L + i] = key;
-    }
-    sbuf[i] = comp;
-  }
-  bitonic_sort_desc(sbuf, P2);
-  for (int t = tid; t < P2; t += kSelThreads)
-    if (sbuf[t] != 0 && (t + 1 == P2 || sbuf[t + 1] == 0)) s_cnt = t + 1;
-  __syncthreads();
-  {
-    const int take = min(max(a.k, 0), s_cnt);
-    for (int t = tid; t < take; t += kSelThreads) {
-      const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
-      flags[idx] = F_SEL | F_MSTAR;
+    for (int i = tid; i < L; i += kSelThreads) {
+      if (!in1[i]) continue;
+      unsigned long long dq = 0;
+      if (!okey)
+        for (int r = 1; r < a.phi_len; ++r) dq += (unsigned long long)(r < kPhiMax ? s_phi[r] : a.phi_q30[r]) * known_at(i, r);
+      finish_key(i, dq, okey ? 0.f : conf[i]);
     }
   }
   __syncthreads();
 
-  // ---- stage 2: top-p over the candidates ----
-  if (tid == 0) s_cnt = 0;
-  for (int j = tid; j < P2; j += kSelThreads) {
-    uint64_t comp = 0;
-    if (j < L) {
-      const bool cand = a.stage2_candidates == 0 ? (smask[j] == 0) : ((flags[j] & F_MSTAR) == 0);
-      if (cand) comp = ((uint64_t)__float_as_uint(clean_score(cs[j])) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)j);
-    }
-    sbuf[j] = comp;
-  }
-  bitonic_sort_desc(sbuf, P2);
-  for (int t = tid; t < P2; t += kSelThreads)
-    if (sbuf[t] != 0 && (t + 1 == P2 || sbuf[t + 1] == 0)) s_cnt = t + 1;
-  __syncthreads();
+  // ---- stage 1: the k largest keys of the set, lower position first among equal keys ----
   {
-    const int ncand = s_cnt;
-    const int per = max(1, P2 / kSelThreads);
-    const int t0 = tid * per;
+    const int take = min(max(a.k, 0), nm);
+    if (take == nm) {
+      for (int i = tid; i < L; i += kSelThreads)
+        if (in1[i]) flags[i] = F_SEL | F_MSTAR;
+    } else if (take > 0 && nm <= kRankMax) {
+      // rank of a listed position = how many others come before it; every thread reads the same entry at a time
+      for (int e = tid; e < nm; e += kSelThreads) {
+        const unsigned long long mine = mlist[e];
+        int rank = 0;
+        for (int f = 0; f < nm; ++f) rank += mlist[f] > mine ? 1 : 0;
+        if (rank < take) flags[0xFFFFFFFFu - (uint32_t)(mine & 0xFFFFFFFFull)] = F_SEL | F_MSTAR;
+      }
+    } else if (take > 0) {
+      const unsigned long long want = (unsigned long long)take;
+      take_until_crossed(kb, L, [&](int j) { return in1[j] != 0; }, [](uint32_t) { return 1ull; },
+                         [&](unsigned long long w) { return w >= want; }, flags, (uint8_t)(F_SEL | F_MSTAR), rsc, 0u, 0xFFFFFFFFu);
+    }
+    __syncthreads();
+  }
+
+  // ---- stage 2: top-p over the candidates by influence score ----
+  if (a.p > 0.f) {
+    const bool mode1 = a.stage2_candidates != 0;
+    auto cand = [&](int j) { return mode1 ? (flags[j] & F_MSTAR) == 0 : smask[j] == 0; };
+    auto mass = [](uint32_t bits) { return (unsigned long long)__double2ull_rd((double)__uint_as_float(bits) * 4294967296.0); };
     unsigned long long local = 0;
-    if (t0 < P2) {
-      for (int e = 0; e < per; ++e) {
-        const float cv = __uint_as_float((uint32_t)(sbuf[t0 + e] >> 32));
-        local += __double2ull_rd((double)cv * 4294967296.0);
-      }
-    }
-    const unsigned long long excl =
-        block_exclusive_scan<unsigned long long>(local, (unsigned long long*)warp_buf64,
-                                                 (unsigned long long*)&s_total64);
-    if (tid == 0) s_take = (a.p > 0.f) ? ncand : 0;
-    __syncthreads();
-    if (a.p > 0.f && t0 < P2) {
-      const double thr = __dmul_rn((double)a.p, __ull2double_rn(s_total64));
-      unsigned long long run = excl;
-      for (int e = 0; e < per; ++e) {
-        const int t = t0 + e;
-        if (t >= ncand) break;
-        const float cv = __uint_as_float((uint32_t)(sbuf[t] >> 32));
-        run += __double2ull_rd((double)cv * 4294967296.0);
-        if (__ull2double_rn(run) > thr) { atomicMin(&s_take, t + 1); break; }
-      }
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+    for (int j = tid; j < L; j += kSelThreads)
+      if (cand(j)) { local += mass(cb[j]); lo = min(lo, cb[j]); hi = max(hi, cb[j]); }
+    for (int o = 16; o > 0; o >>= 1) local += shfl_xor_u64(local, o);
+    lo = __reduce_min_sync(0xffffffffu, lo); hi = __reduce_max_sync(0xffffffffu, hi);
+    if (lane == 0) {
+      if (local) atomicAdd(&s_mass, local);
+      atomicMin(&s_lo, lo); atomicMax(&s_hi, hi);
     }
     __syncthreads();
-    const int take = s_take;
-    for (int t = tid; t < take; t += kSelThreads) {
-      const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sbuf[t] & 0xFFFFFFFFull);
-      flags[idx] |= F_SEL;
-    }
-  }
-  __syncthreads();
-
+    const double thr = __dmul_rn((double)a.p, __ull2double_rn(s_mass));
+    take_until_crossed(cb, L, cand, mass, [&](unsigned long long w) { return __ull2double_rn(w) > thr; }, flags, (uint8_t)F_SEL, rsc,
+                       s_lo, max(s_hi, s_lo));
   }
 
   // ---- forced rows ----
@@ -352,14 +401,12 @@ int launch_select(const SelectArgs& a, cudaStream_t st) {
   if (a.batch <= 0) return D2C_OK;
   // a sequence of 65535 selected rows would overflow the packed 16-bit counters
   if (a.seq_len > 8192) { set_global_error("select: seq_len %d > 8192", a.seq_len); return D2C_ECAPACITY; }
-  int P2 = 32;
-  while (P2 < a.seq_len) P2 <<= 1;
-  const size_t smem = (size_t)P2 * 8 + 2 * (size_t)a.seq_len;
+  const size_t smem = (size_t)a.seq_len * 11;               // two 32-bit words and three flag bytes per position
   static PerDevice attr_set;
   if (attr_set.first()) {
-    D2C_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8192 * 8 + 2 * 8192));
+    D2C_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8192 * 11));
   }
-  D2C_LAUNCH((select_kernel), a.batch, kSelThreads, smem, st, a, P2);
+  D2C_LAUNCH((select_kernel), a.batch, kSelThreads, smem, st, a);
   if (a.batch > 1) {
     dim3 grid(ceil_div(a.seq_len, 256), a.batch);
     D2C_LAUNCH((select_finalize_kernel), grid, 256, 0, st, a);
