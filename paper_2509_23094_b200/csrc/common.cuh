@@ -117,8 +117,8 @@ struct GemmArgs {
   // the QKV projection; C/ldc is the QKV activation buffer (only its Q part is written)
   const int32_t* q_sel_idx; const int32_t* q_row_seq; const float2* q_rope; bf16* q_kc; bf16* q_vc;
   int q_cache_seq, q_hq, q_hkv, q_dh;
-  // split-K scratch of the one-SM tcgen05 kernel (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
-  // and as many zero-initialised arrival counters
+  // split-K scratch of the tcgen05 kernels (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
+  // and twice as many zero-initialised counters
   float* sk_partials; int32_t* sk_counters; int sk_max_tiles;
   // optional (tcgen05 kernels): CTA 0 stores {clock64, globaltimer ns} at its start and its end, which gives the
   // SM clock the launch really ran at (a power-capped clock is not what a coarse NVML sample shows)

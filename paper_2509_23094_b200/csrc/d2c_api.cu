@@ -86,7 +86,7 @@ static size_t carve(const d2c_config& c, void* base, Buffers* out) {
   b.st_max = w.take<float>(R * nt); b.st_sum = w.take<float>(R * nt); b.st_arg = w.take<int32_t>(R * nt);
   b.u0 = w.take<float>(R); b.u1 = w.take<float>(R);
   b.partial = w.take<float>((size_t)kRolloutSplit * R + (R + 3) / 4);     // partial sums + selected-flag bytes
-  b.sk_partials = w.take<float>((size_t)kSkMaxTiles * 128 * 256); b.sk_counters = w.take<int32_t>(kSkMaxTiles);
+  b.sk_partials = w.take<float>((size_t)kSkMaxTiles * 128 * 256); b.sk_counters = w.take<int32_t>(2 * kSkMaxTiles);     // arrival and done counters
   b.gemm_clocks = w.take<long long>(4);
   // scratch for the head-split of the abar kernel: only worth having when the (rows x keys) grid is small
   const size_t tiles_worst = (size_t)ceil_div((int)L, 128) * ceil_div((int)L, 128) * B;

@@ -59,42 +59,51 @@ __device__ __forceinline__ uint4 epi_pack(const float (&f)[8]) {
 }
 
 // C[row][n0 .. n0 + out_cols) = acc (+ bias) or C += acc.  load_chunk(col, v) must deliver accumulator columns
-// [col, col + 32) of the calling lane's row and must be called by the whole warp.
+// [col, col + 32) of the calling lane's row and must be called by the whole warp.  Only the 32-column chunks
+// [c_begin, c_end) of the tile are handled (c_end < 0: all of them), which lets the parts of a split-K tile
+// share one tile's epilogue.
 template <int EPI, typename LoadChunk>
-__device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int out_cols) {
-  const int pairs = out_cols >> 6;                            // 64 output columns per pass
+__device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int out_cols,
+                                              int c_begin = 0, int c_end = -1) {
+  if (c_end < 0) c_end = out_cols >> 5;
+  const int passes = (c_end - c_begin + 1) >> 1;              // up to 64 output columns per pass
   const bool vec = (g.ldc & 7) == 0;
   const int rsub = w.lane >> 2, cg = w.lane & 3;
   uint4 rc[8], rn[8];                                         // residual of this pass and of the next one
   auto load_res = [&](int p, uint4 (&r)[8]) {
-    if (EPI == EPI_RESIDUAL && vec && p < pairs) {
+    if (EPI == EPI_RESIDUAL && vec && p < passes) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const int row = w.row0 + j * 8 + rsub, col = n0 + p * 64 + h * 32 + cg * 8;
-          if (row < w.n && col + 8 <= g.N) r[j * 2 + h] = __ldcg(reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col));
+          const int row = w.row0 + j * 8 + rsub, col = n0 + (c_begin + 2 * p + h) * 32 + cg * 8;
+          if (row < w.n && c_begin + 2 * p + h < c_end && col + 8 <= g.N)
+            r[j * 2 + h] = __ldcg(reinterpret_cast<const uint4*>(g.C + (size_t)row * g.ldc + col));
         }
     }
   };
   load_res(0, rc);
 #pragma unroll 1
-  for (int p = 0; p < pairs; ++p) {
+  for (int p = 0; p < passes; ++p) {
     load_res(p + 1, rn);
+    const int c0 = c_begin + 2 * p;
+    const bool two = c0 + 1 < c_end;
     {
       uint32_t v[32];
-      load_chunk(p * 64, v);
+      load_chunk(c0 * 32, v);
       epi_stage_put(w, 0, v);
-      load_chunk(p * 64 + 32, v);
-      epi_stage_put(w, 1, v);
+      if (two) {
+        load_chunk(c0 * 32 + 32, v);
+        epi_stage_put(w, 1, v);
+      }
     }
     __syncwarp();
 #pragma unroll
     for (int j = 0; j < 4; ++j)
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        const int row = w.row0 + j * 8 + rsub, col = n0 + p * 64 + h * 32 + cg * 8;
-        if (row >= w.n || col >= g.N) continue;
+        const int row = w.row0 + j * 8 + rsub, col = n0 + (c0 + h) * 32 + cg * 8;
+        if (row >= w.n || col >= g.N || (h == 1 && !two)) continue;
         float f[8];
         epi_stage_get(w, h, j * 8 + rsub, cg, f);
         bf16* dst = g.C + (size_t)row * g.ldc + col;
@@ -127,13 +136,15 @@ __device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const Gemm
 }
 
 // C[row][n0 .. n0 + oc) = silu(gate) * up, gate in accumulator columns [0, oc) and up in [oc, 2 oc); oc is a
-// multiple of 32.
+// multiple of 32.  Handles the 32-column chunks [c_begin, c_end) of the oc outputs (c_end < 0: all).
 template <typename LoadChunk>
-__device__ __forceinline__ void epilogue_swiglu(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int oc) {
+__device__ __forceinline__ void epilogue_swiglu(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int oc,
+                                                int c_begin = 0, int c_end = -1) {
+  if (c_end < 0) c_end = oc >> 5;
   const bool vec = (g.ldc & 7) == 0;
   const int rsub = w.lane >> 2, cg = w.lane & 3;
 #pragma unroll 1
-  for (int c = 0; c < (oc >> 5); ++c) {
+  for (int c = c_begin; c < c_end; ++c) {
     {
       uint32_t v[32];
       load_chunk(c * 32, v);
@@ -170,10 +181,13 @@ __device__ __forceinline__ void epilogue_swiglu(LoadChunk&& load_chunk, const Ge
 // Fused epilogue of the QKV projection: bias, rotary embedding of the Q and K heads at the row's absolute
 // position, Q written to the activation buffer, K and V written straight into the layer's cache row of
 // (sequence, position).  The rotation pairs column i of a head with column i + Dh/2: the two 32-column
-// chunks of a pass are the matching pieces of the lower and the upper half head.
+// chunks of a pass are the matching pieces of the lower and the upper half head.  The tile's passes are numbered
+// head by head (out_cols / 64 of them); only passes [u_begin, u_end) are handled (u_end < 0: all).
 template <typename LoadChunk>
-__device__ __forceinline__ void epilogue_qkv_rope(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int out_cols) {
+__device__ __forceinline__ void epilogue_qkv_rope(LoadChunk&& load_chunk, const GemmArgs& g, const EpiWarp& w, int n0, int out_cols,
+                                                  int u_begin = 0, int u_end = -1) {
   const int dh = g.q_dh, half_chunks = dh >> 6;               // 32-column chunks per half head: 1 (Dh 64) or 2 (Dh 128)
+  if (u_end < 0) u_end = out_cols >> 6;
   const int rsub = w.lane >> 2, cg = w.lane & 3;
   int pos[4];
   size_t cache_row[4];
@@ -193,6 +207,8 @@ __device__ __forceinline__ void epilogue_qkv_rope(LoadChunk&& load_chunk, const 
     const bool is_q = head < g.q_hq, is_k = !is_q && head < g.q_hq + g.q_hkv;
 #pragma unroll 1
     for (int c = 0; c < half_chunks; ++c) {
+      const int unit = hc * half_chunks + c;
+      if (unit < u_begin || unit >= u_end) continue;          // uniform across the warp
       const int lc = hc * (dh >> 5) + c;
       {
         uint32_t v[32];

@@ -67,7 +67,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
   __shared__ __align__(8) uint64_t bars[2 * ST_MAX + 4];     // full[], empty[], acc_full[2], acc_empty[2]
   __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag, sk_last;
+  __shared__ int abort_flag;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (ST_MAX + s); };
@@ -99,10 +99,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   const bool sk_ok = g.sk_partials != nullptr && g.sk_counters != nullptr;
   // Split-K for launches with fewer tiles than SMs (few live rows: the launch streams weights and every
   // idle SM is lost bandwidth): each tile's K range is cut into S equal parts of at least four k-blocks,
-  // handled by different CTAs.  Parts park their fp32 accumulators in scratch; the part that arrives last
-  // adds them in part order (no waiting, deterministic) and runs the epilogue.
+  // one (tile, part) item per CTA at most, so all parts of a tile run at the same time.  Parts park their fp32
+  // accumulators in scratch and meet at a counter (a bounded wait); then each part adds, in part order
+  // (deterministic), the partial sums of its own share of the tile's columns and runs the epilogue on them,
+  // so the reduction and the epilogue are spread over S CTAs instead of falling on one.
   auto split_of = [&](int tiles) {
-    if (!sk_ok || tiles <= 0 || tiles >= G) return 1;
+    if (!sk_ok || EPI == EPI_LMSTATS || tiles <= 0 || tiles >= G) return 1;
     const int s = max(1, min(min(G / tiles, KT / 4), kSkMaxParts));
     return tiles * s <= g.sk_max_tiles ? s : 1;
   };
@@ -131,9 +133,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   const int a_rows_max = n >= 128 ? 128 : (n > 64 ? 128 : (n > 32 ? 64 : 32));
   const int b_rows = (EPI == EPI_SWIGLU) ? ACC_COLS : bn;
   const int sub_bytes = ((a_rows_max + b_rows) * TK * 2 + 1023) & ~1023;
-  const int stage_bytes = KSUB * sub_bytes;
+  const int ring_bytes = ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2;
+  // two k-blocks per stage halve the issuing thread's barrier round-trips, but a ring of only two such stages
+  // leaves one stage in flight while the other is consumed: big boxes (few-row weight streaming) keep one
+  // k-block per stage and so twice as many stages
+  const int ksub = ring_bytes / (KSUB * sub_bytes) >= 3 ? KSUB : 1;
+  const int stage_bytes = ksub * sub_bytes;
   // the MMA always reads 128 rows of A: keep that read inside the allocation when the A box is smaller
-  const int nst = min(ST_MAX, (ST * STAGE_BYTES - (128 - a_rows_max) * TK * 2) / stage_bytes);
+  const int nst = min(ST_MAX, ring_bytes / stage_bytes);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -147,9 +154,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         const int rows = n - m0;                              // live rows of this tile: load no more than needed
         const CUtensorMap* ma = rows <= 32 ? &tmA32 : (rows <= 64 ? &tmA64 : &tmA128);
         const uint32_t kb_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2 + (uint32_t)b_rows * TK * 2;
-        for (int kt = k0; kt < k1; kt += KSUB, ++it) {
+        for (int kt = k0; kt < k1; kt += ksub, ++it) {
           const int s = it % nst;
-          const int nsub = min(KSUB, k1 - kt);
+          const int nsub = min(ksub, k1 - kt);
           if (!mbar_wait(empty_bar(s), ((it / nst) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
 #pragma unroll
@@ -193,8 +200,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 4)) { ok = false; break; }
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
-        for (int j = 0; j < nk; j += KSUB) {
-          const int nsub = min(KSUB, nk - j);
+        for (int j = 0; j < nk; j += ksub) {
+          const int nsub = min(ksub, nk - j);
           if (!mbar_wait(full_bar(st), ph, abortp, status, 2)) { ok = false; break; }
           tc_fence_after();
           const uint64_t adesc = desc0 + (uint64_t)(st * (stage_bytes >> 4)), bdesc = adesc + b_off;
@@ -256,16 +263,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (warp == 2 && lane == 0) {
           mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf)); mbar_arrive(acc_empty(buf));
-          const int old = atomicAdd(&g.sk_counters[tile], 1);
-          const int last = (old == S - 1) ? 1 : 0;
-          if (last) g.sk_counters[tile] = 0;                 // every part has arrived: ready for the next launch
-          sk_last = last;
+          atomicAdd(&g.sk_counters[tile], 1);
+          // every other part of this tile is running on another SM: wait (bounded) until all have parked their sums
+          const long long t0 = clock64();
+          volatile int32_t* cnt = g.sk_counters + tile;
+          while (*cnt < S) {
+            if (*abortp) break;
+            if (clock64() - t0 > kWaitCycles) {
+              *abortp = 1;
+              if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = 5;
+              break;
+            }
+          }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        reduce = sk_last != 0;
-        asm volatile("bar.sync 1, 128;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
-        if (!reduce) continue;
+        if (*abortp) break;
         __threadfence();
+        reduce = true;
       }
       auto load_chunk = [&](int col, uint32_t (&v)[32]) {     // 32 accumulator columns of this thread's row
         if (!reduce) {
@@ -298,12 +312,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         }
       };
       const EpiWarp ew{smem_base + (uint32_t)(ST * STAGE_BYTES) + (uint32_t)(quarter * kEpiStageBytes), m0 + quarter * 32, n, lane};
+      // a split-K part finishes its share of the tile's epilogue passes; an unsplit tile all of them
+      const int units = (EPI == EPI_STORE || EPI == EPI_RESIDUAL) ? OUT_COLS >> 5 : (EPI == EPI_SWIGLU ? OUT_COLS >> 5 : OUT_COLS >> 6);
+      const int u0 = reduce ? part * units / S : 0, u1 = reduce ? (part + 1) * units / S : units;
       if (EPI == EPI_QKV_ROPE) {
-        epilogue_qkv_rope(load_chunk, g, ew, n0, OUT_COLS);
+        epilogue_qkv_rope(load_chunk, g, ew, n0, OUT_COLS, u0, u1);
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-        epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS);
+        epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS, u0, u1);
       } else if (EPI == EPI_SWIGLU) {
-        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS);
+        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS, u0, u1);
       } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
         for (int half = 0; half < bn / 128; ++half) {         // statistics are kept per 128 columns
@@ -340,6 +357,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
             const size_t o = (size_t)row * g.n_tiles + stile;
             g.st_max[o] = mx; g.st_sum[o] = sum; g.st_arg[o] = arg;
           }
+        }
+      }
+      if (reduce) {
+        // the part that finishes reading last puts both counters back for the next launch
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          const int old = atomicAdd(&g.sk_counters[g.sk_max_tiles + tile], 1);
+          if (old == S - 1) { g.sk_counters[tile] = 0; g.sk_counters[g.sk_max_tiles + tile] = 0; }
         }
       }
       // hand the accumulator back to the MMA warp (a split-K part has done so already)

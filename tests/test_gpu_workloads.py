@@ -204,6 +204,28 @@ def test_llada_single_layer_row_counts_around_the_pair_tile(n_sel):
     assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
 
 
+@pytest.mark.parametrize("n_sel", [1, 33, 64, 100, 128])
+def test_llada_single_layer_few_forced_rows(n_sel):
+    """At most 128 rows: from the second such step on the projections run on the one-SM kernel, every tile's K
+    range split over several SMs whose parts each finish a share of the tile's columns."""
+    wl = inputs.WORKLOADS["llada1l_1024"]
+    r = Runner(wl)
+    B, L = wl.batch, wl.seq_len
+    r.step(10 ** 6, 1.0)
+    rng = np.random.default_rng(1000 + n_sel)
+    for rep in range(2):
+        forced = [sorted(rng.choice(L, n_sel, replace=False).tolist())]
+        kc0 = r.ctx.view("kcache").clone(); vc0 = r.ctx.view("vcache").clone()
+        ro, S = r.step(0, 0.0, forced=forced)
+        torch.cuda.synchronize()
+        assert len(S[0]) == n_sel
+        r.check_layers(ro, S, [0], rows_per_seq=64, seqs=[0], seed=n_sel + rep)
+        r.check_lm_head()
+        kc1 = r.ctx.view("kcache"); vc1 = r.ctx.view("vcache")
+        keep = torch.ones(L, dtype=torch.bool, device="cuda"); keep[torch.from_numpy(S[0]).cuda()] = False
+        assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
+
+
 def test_llada_32_layers_768_with_a_committed_token():
     r, ro, S, _ = _run("llada_decode", [0, 1, 16, 31], [0, 31], [0])
     # decode-loop shape: commit the most confident masked row, force it into the next step
