@@ -158,12 +158,12 @@ def aggregate_replicas(total_ms, e2e_s, rows, world, device):
     return float(tmax[0]), float(tmax[1]), float(tsum[2])
 
 
-def build_pair(wl, device, rollout_layers=0):
+def build_pair(wl, device, rollout_layers=0, flags=0):
     from paper_2509_23094_b200 import binding
     w_cpu = inputs.make_weights(wl.shape, seed=wl.seed, device=device if wl.shape.n_layers > 4 else "cpu")
     w_dev = {"layers": [{k: (None if v is None else v.to(device)) for k, v in lyr.items()} for lyr in w_cpu["layers"]],
              "g_final": w_cpu["g_final"].to(device), "w_lm": w_cpu["w_lm"].to(device), "embed": w_cpu["embed"].to(device)}
-    cfg = binding.make_config(wl.shape, wl.batch, wl.seq_len, sigma=wl.sigma, rollout_layers=rollout_layers)
+    cfg = binding.make_config(wl.shape, wl.batch, wl.seq_len, sigma=wl.sigma, rollout_layers=rollout_layers, flags=flags)
     ctx = binding.Context(cfg, w_dev, device=device)
     mask = inputs.make_mask(wl)
     tokens = inputs.make_tokens(wl, mask)
@@ -177,7 +177,7 @@ def run_ours(args, rank, world, device):
         from dataclasses import replace as _replace
         wl = _replace(wl, p=wl.p if args.p is None else args.p, k=wl.k if args.k is None else args.k)
     shape, B, L, d = wl.shape, wl.batch, wl.seq_len, wl.shape.d_model
-    w_cpu, w_dev, ctx, mask, tokens, h0 = build_pair(wl, device, args.rollout_layers)
+    w_cpu, w_dev, ctx, mask, tokens, h0 = build_pair(wl, device, args.rollout_layers, args.flags)
     mask_dev = mask.to(device)
     stream = torch.cuda.current_stream()
 
@@ -506,6 +506,7 @@ def main():
     ap.add_argument("--k", type=int, default=None, help="override the workload's k")
     ap.add_argument("--rollout-layers", type=int, default=0,
                     help="roll the attention out over the first n layers only (the paper's Rollout-5 variant); 0 = all layers")
+    ap.add_argument("--flags", type=int, default=0, help="D2C_FLAG_* bits for the context (kernel variants kept as cross-checks)")
     ap.add_argument("--no-extras", action="store_true", help="skip the labelled extra run at the paper's default p = 0.1")
     ap.add_argument("--scores", default="rollout", choices=["rollout", "zipf"],
                     help="stage-2 scores before each timed step: the prefill's rollout (default) or a seeded Zipf(1.0)")

@@ -77,6 +77,9 @@ typedef struct {
 #define D2C_FLAG_PORTABLE_ATTENTION 2   /* same for the attention kernels                                                */
 #define D2C_FLAG_ONE_SM_GEMM 4          /* keep the GEMMs on the one-SM tcgen05 kernel (no CTA pairs)                    */
 #define D2C_FLAG_SERIAL 8               /* enqueue every kernel of a step on the caller's stream, one after the other    */
+#define D2C_FLAG_FOLDED_NORMS 16        /* fold the layers' RMSNorms into the GEMM epilogues around them (x * gain and the row's sums of
+                                           squares written by the residual epilogue, the row scale applied by the next projection)
+                                           instead of running them as kernels of their own; measured slower at every workload          */
 
 /* Weights.  The arrays of per-layer pointers are HOST arrays of n_layers DEVICE
  * pointers; they are copied at create, the device memory is borrowed for the

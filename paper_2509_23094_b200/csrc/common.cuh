@@ -120,6 +120,14 @@ struct GemmArgs {
   // split-K scratch of the tcgen05 kernels (null: no split): sk_max_tiles partial tiles of 128 x 256 fp32
   // and twice as many zero-initialised counters
   float* sk_partials; int32_t* sk_counters; int sk_max_tiles;
+  // RMSNorm folded into the GEMMs around it (tcgen05 kernels).  A residual epilogue that is given nx_out also writes
+  // nx_out[row][col] = bf16(x_new[row][col] * nx_gain[col]) (same leading dimension as C) and, per (row, 32-column
+  // chunk), the sum of squares of the new x into nx_ssq[row][N / 32].  A GEMM that is given in_ssq (K / 32 such
+  // partial sums per row of A) multiplies accumulator row r by rsqrt(sum_t in_ssq[r][t] / K + in_eps) before its
+  // own epilogue: the per-row scalar commutes with the contraction, so A = x * gain gives the same product as
+  // A = rmsnorm(x) * gain.
+  bf16* nx_out; const bf16* nx_gain; float* nx_ssq;
+  const float* in_ssq; float in_eps;
   // optional (tcgen05 kernels): CTA 0 stores {clock64, globaltimer ns} at its start and its end, which gives the
   // SM clock the launch really ran at (a power-capped clock is not what a coarse NVML sample shows)
   long long* clock_probe;

@@ -51,7 +51,7 @@ struct Buffers {
   bf16 *kcache, *vcache; float *conf, *c, *key; int32_t *pred, *status;
   int32_t *sel_idx, *row_seq, *row_off, *lm_rows, *lm_off, *slot_of_pos, *rank_s, *rank_lm, *n_b, *nm_b;
   uint32_t* phi; float2* rope;
-  bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar;
+  bf16 *x, *xn, *qkv, *o, *hmid, *xm; float *lse, *abar, *ssq;
   float *st_max, *st_sum; int32_t* st_arg;
   float *u0, *u1, *partial;
   float* sk_partials; int32_t* sk_counters; long long* gemm_clocks;
@@ -81,6 +81,7 @@ static size_t carve(const d2c_config& c, void* base, Buffers* out) {
   b.x = w.take<bf16>(R * d); b.xn = w.take<bf16>(R * d); b.qkv = w.take<bf16>(R * qkv_out);
   b.o = w.take<bf16>(R * (size_t)c.n_q_heads * c.head_dim); b.hmid = w.take<bf16>(R * (size_t)c.d_ffn);
   b.xm = w.take<bf16>(R * d); b.lse = w.take<float>(R * (size_t)c.n_q_heads);
+  b.ssq = w.take<float>(R * (d / 32));                      // per (row, 32 columns): sum of squares of the residual stream
   b.abar = w.take<float>((size_t)rollout_depth(c) * R * L);
   const size_t nt = lm_tiles(c.vocab);
   b.st_max = w.take<float>(R * nt); b.st_sum = w.take<float>(R * nt); b.st_arg = w.take<int32_t>(R * nt);
@@ -110,7 +111,7 @@ static const char* check_config(const d2c_config* c) {
   if (c->max_batch < 1 || c->max_seq < 1 || c->max_seq > 8192) return "max_batch >= 1 and 1 <= max_seq <= 8192 required";
   if (!(c->rope_base > 1.f) || !(c->rms_eps >= 0.f) || !(c->sigma > 0.f)) return "rope_base > 1, rms_eps >= 0, sigma > 0 required";
   if (c->stage2_candidates != 0 && c->stage2_candidates != 1) return "stage2_candidates must be 0 or 1";
-  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION | D2C_FLAG_ONE_SM_GEMM | D2C_FLAG_SERIAL))) return "rollout_layers >= 0 and no unknown flag bits required";
+  if (c->rollout_layers < 0 || (c->flags & ~(D2C_FLAG_PORTABLE_GEMM | D2C_FLAG_PORTABLE_ATTENTION | D2C_FLAG_ONE_SM_GEMM | D2C_FLAG_SERIAL | D2C_FLAG_FOLDED_NORMS))) return "rollout_layers >= 0 and no unknown flag bits required";
   return nullptr;
 }
 
@@ -422,13 +423,28 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
   D2C_TRY(ctx, mark(ctx, PH_GATHER));
   D2C_TRY(ctx, launch_gather_norm((const bf16*)a->h0, b.sel_idx, b.row_seq, n_rows, R, L, d, ctx->g_attn[0], c.rms_eps, x, b.xn, st));
   const int depth = rollout_depth(c);
+  // on request the RMSNorms inside the layers ride in the tcgen05 GEMMs' epilogues (all four projections must run on
+  // those kernels).  Off by default: the longer epilogues and the row scaling cost the GEMMs more than the two small
+  // kernels per layer take (8.7 -> 9.2 ms per step at 488 rows x 32 layers, 420 -> 434 ms at 8 x 4096).
+  bool fold = (c.flags & D2C_FLAG_FOLDED_NORMS) && !(c.flags & D2C_FLAG_PORTABLE_GEMM);
+  {
+    const int shapes[4][2] = {{qkv_out, d}, {d, hq * dh}, {c.d_ffn, d}, {d, c.d_ffn}};       // {N, K}
+    const bf16* as[4] = {b.xn, b.o, b.xn, b.hmid};
+    for (int i = 0; i < 4 && fold; ++i) {
+      GemmArgs t{};
+      t.A = as[i]; t.lda = shapes[i][1]; t.W = ctx->wqkv[0]; t.max_rows = R; t.N = shapes[i][0]; t.K = shapes[i][1];
+      fold = gemm_tc_supported(t) && (d & 7) == 0;
+    }
+  }
   for (int l = 0; l < c.n_layers; ++l) {
     if (out && out->layer_in) {
       cudaError_t e = cudaMemcpyAsync(static_cast<bf16*>(out->layer_in) + (size_t)l * R * d, x, (size_t)R * d * sizeof(bf16),
                                       cudaMemcpyDeviceToDevice, st);
       if (e != cudaSuccess) return fail(ctx, D2C_ECUDA, "d2c_step: %s", cudaGetErrorString(e));
     }
-    if (l > 0) {
+    // RMSNorm folded into the projections (tcgen05 GEMMs): the residual epilogue before a norm leaves x * gain in xn
+    // and the row's sums of squares in ssq, the projection after it scales its accumulator rows by rsqrt(mean + eps)
+    if (l > 0 && !fold) {
       D2C_TRY(ctx, mark(ctx, PH_NORM));
       D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_attn[l], c.rms_eps, b.xn, st));
     }
@@ -440,6 +456,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     GemmArgs g{};
     g.A = b.xn; g.lda = d; g.W = ctx->wqkv[l]; g.bias = ctx->bqkv[l]; g.C = b.qkv; g.ldc = qkv_out;
     g.n_rows = n_rows; g.max_rows = R; g.N = qkv_out; g.K = d;
+    if (fold && l > 0) { g.in_ssq = b.ssq; g.in_eps = c.rms_eps; }
     bf16* kc = b.kcache + (size_t)l * cache_layer; bf16* vc = b.vcache + (size_t)l * cache_layer;
     if (!(c.flags & D2C_FLAG_PORTABLE_GEMM) && gemm_tc_supported(g)) {
       // QKV projection with bias, rotary embedding and the K/V scatter in its epilogue
@@ -486,17 +503,22 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     D2C_TRY(ctx, mark(ctx, PH_O));
     GemmArgs go{};
     go.A = b.o; go.lda = hq * dh; go.W = ctx->wo[l]; go.C = x; go.ldc = d; go.n_rows = n_rows; go.max_rows = R; go.N = d; go.K = hq * dh;
+    if (fold) { go.nx_out = b.xn; go.nx_gain = ctx->g_ffn[l]; go.nx_ssq = b.ssq; }
     D2C_TRY(ctx, gemm(ctx, go, EPI_RESIDUAL));
-    D2C_TRY(ctx, mark(ctx, PH_NORM));
-    D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_ffn[l], c.rms_eps, b.xn, st));
+    if (!fold) {
+      D2C_TRY(ctx, mark(ctx, PH_NORM));
+      D2C_TRY(ctx, launch_rmsnorm(x, nullptr, n_rows, R, d, ctx->g_ffn[l], c.rms_eps, b.xn, st));
+    }
     D2C_TRY(ctx, mark(ctx, PH_GATEUP));
     GemmArgs gf{};
     gf.A = b.xn; gf.lda = d; gf.W = ctx->w_gate[l]; gf.W2 = ctx->w_up[l]; gf.C = b.hmid; gf.ldc = c.d_ffn;
     gf.n_rows = n_rows; gf.max_rows = R; gf.N = c.d_ffn; gf.K = d;
     gf.clock_probe = ctx->prof ? b.gemm_clocks : nullptr;
+    if (fold) { gf.in_ssq = b.ssq; gf.in_eps = c.rms_eps; }
     D2C_TRY(ctx, gemm(ctx, gf, EPI_SWIGLU));
     GemmArgs gd{};
     gd.A = b.hmid; gd.lda = c.d_ffn; gd.W = ctx->w_down[l]; gd.C = x; gd.ldc = d; gd.n_rows = n_rows; gd.max_rows = R; gd.N = d; gd.K = c.d_ffn;
+    if (fold && l + 1 < c.n_layers) { gd.nx_out = b.xn; gd.nx_gain = ctx->g_attn[l + 1]; gd.nx_ssq = b.ssq; }
     D2C_TRY(ctx, mark(ctx, PH_DOWN));
     D2C_TRY(ctx, gemm(ctx, gd, EPI_RESIDUAL));
   }

@@ -23,6 +23,26 @@ struct EpiWarp {
 
 union EpiPack8 { uint4 u; __nv_bfloat162 h[4]; };
 
+// rsqrt(mean(x^2) + eps) of row `row` of the A operand, from the K / 32 partial sums of squares the GEMM that wrote
+// x left behind (added here in chunk order: deterministic); 1 when the launch carries no folded RMSNorm.
+__device__ __forceinline__ float folded_row_scale(const GemmArgs& g, int row, bool row_ok) {
+  if (!g.in_ssq) return 1.f;
+  float s = 0.f;
+  if (row_ok) {
+    const int chunks = g.K >> 5;
+    const float* sp = g.in_ssq + (size_t)row * chunks;
+    if ((chunks & 3) == 0) {
+      for (int t = 0; t < chunks; t += 4) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(sp + t));
+        s += (v.x + v.y) + (v.z + v.w);
+      }
+    } else {
+      for (int t = 0; t < chunks; ++t) s += __ldcg(sp + t);
+    }
+  }
+  return rsqrtf(s / (float)g.K + g.in_eps);
+}
+
 // Row `lane` of sub-tile `half` <- the 32 columns in v.  16-byte pieces are XOR-swizzled with the row so that
 // neither this write (same piece, 32 rows) nor the transposed read (same row, 4 lanes) conflicts on banks.
 __device__ __forceinline__ void epi_stage_put(const EpiWarp& w, int half, const uint32_t (&v)[32]) {
@@ -103,30 +123,52 @@ __device__ __forceinline__ void epilogue_rows(LoadChunk&& load_chunk, const Gemm
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int row = w.row0 + j * 8 + rsub, col = n0 + (c0 + h) * 32 + cg * 8;
-        if (row >= w.n || col >= g.N || (h == 1 && !two)) continue;
-        float f[8];
-        epi_stage_get(w, h, j * 8 + rsub, cg, f);
-        bf16* dst = g.C + (size_t)row * g.ldc + col;
-        if (vec && col + 8 <= g.N) {
-          if (EPI == EPI_RESIDUAL) {
-            EpiPack8 old; old.u = rc[j * 2 + h];
+        const bool live = row < w.n && col < g.N && (h == 0 || two);
+        float sq = 0.f;                                       // this lane's share of the row's sum of squares in the chunk
+        if (live) {
+          float f[8];
+          epi_stage_get(w, h, j * 8 + rsub, cg, f);
+          bf16* dst = g.C + (size_t)row * g.ldc + col;
+          if (vec && col + 8 <= g.N) {
+            if (EPI == EPI_RESIDUAL) {
+              EpiPack8 old; old.u = rc[j * 2 + h];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { const float2 of = __bfloat1622float2(old.h[e]); f[2 * e] += of.x; f[2 * e + 1] += of.y; }
-          } else if (g.bias) {
+              for (int e = 0; e < 4; ++e) { const float2 of = __bfloat1622float2(old.h[e]); f[2 * e] += of.x; f[2 * e + 1] += of.y; }
+            } else if (g.bias) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] += __bfloat162float(g.bias[col + e]);
-          }
-          *reinterpret_cast<uint4*>(dst) = epi_pack(f);
-        } else {
+              for (int e = 0; e < 8; ++e) f[e] += __bfloat162float(g.bias[col + e]);
+            }
+            EpiPack8 xr; xr.u = epi_pack(f);
+            *reinterpret_cast<uint4*>(dst) = xr.u;
+            if (EPI == EPI_RESIDUAL && g.nx_out) {
+              // the next RMSNorm, folded: x * gain for the next GEMM, and the row's sum of squares, both from the stored bf16 x
+              EpiPack8 gn, o; gn.u = __ldg(reinterpret_cast<const uint4*>(g.nx_gain + col));
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            if (col + e < g.N) {
-              float x = f[e];
-              if (EPI == EPI_RESIDUAL) x += __bfloat162float(dst[e]);
-              else if (g.bias) x += __bfloat162float(g.bias[col + e]);
-              dst[e] = __float2bfloat16_rn(x);
+              for (int e = 0; e < 4; ++e) {
+                const float2 xv = __bfloat1622float2(xr.h[e]), gv = __bfloat1622float2(gn.h[e]);
+                sq += xv.x * xv.x + xv.y * xv.y;
+                o.h[e] = __floats2bfloat162_rn(xv.x * gv.x, xv.y * gv.y);
+              }
+              *reinterpret_cast<uint4*>(g.nx_out + (size_t)row * g.ldc + col) = o.u;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              if (col + e < g.N) {
+                float x = f[e];
+                if (EPI == EPI_RESIDUAL) x += __bfloat162float(dst[e]);
+                else if (g.bias) x += __bfloat162float(g.bias[col + e]);
+                dst[e] = __float2bfloat16_rn(x);
+              }
             }
           }
+        }
+        if (EPI == EPI_RESIDUAL && g.nx_ssq) {
+          // the four lanes that share a row add their parts in a fixed order; one of them stores the chunk's sum
+          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+          if (cg == 0 && row < w.n && (h == 0 || two) && n0 + (c0 + h) * 32 < g.N)
+            g.nx_ssq[(size_t)row * (size_t)(g.N >> 5) + (size_t)((n0 >> 5) + c0 + h)] = sq;
         }
       }
     __syncwarp();                                             // the staging buffer is rewritten by the next pass

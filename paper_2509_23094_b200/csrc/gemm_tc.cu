@@ -231,6 +231,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
       const int m0 = (tile % MT) * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
+      const float rscale = folded_row_scale(g, row, row_ok);     // RMSNorm of the A rows folded into this GEMM (1 if none)
       // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
       const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 3));
       if (S > 1) {
@@ -285,6 +286,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
         if (!reduce) {
           tmem_ld32(tbase + col, v);
           tmem_ld_wait();
+          if (g.in_ssq) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * rscale);
+          }
         } else {
           const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + (size_t)(tile * S) * (TM * ACC_COLS)) +
                              (size_t)(col >> 2) * TM + lrow;
@@ -306,8 +311,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
           }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            v[4 * q] = __float_as_uint(acc[q].x); v[4 * q + 1] = __float_as_uint(acc[q].y);
-            v[4 * q + 2] = __float_as_uint(acc[q].z); v[4 * q + 3] = __float_as_uint(acc[q].w);
+            v[4 * q] = __float_as_uint(acc[q].x * rscale); v[4 * q + 1] = __float_as_uint(acc[q].y * rscale);
+            v[4 * q + 2] = __float_as_uint(acc[q].z * rscale); v[4 * q + 3] = __float_as_uint(acc[q].w * rscale);
           }
         }
       };

@@ -230,6 +230,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
+      const float rscale = folded_row_scale(g, row, row_ok);     // RMSNorm of the A rows folded into this GEMM (1 if none)
       // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
       const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 33));
       if (S > 1) {
@@ -278,6 +279,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (!reduce) {
           tmem_ld32(tbase + col, v);
           tmem_ld_wait();
+          if (g.in_ssq) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * rscale);
+          }
         } else {
           float4 t[4][8];
           const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + ((size_t)(tile * S) * 2 + rank) * slot_floats) +
@@ -292,8 +297,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             float4 acc = t[0][q];
 #pragma unroll
             for (int c2 = 1; c2 < 4; ++c2) { acc.x += t[c2][q].x; acc.y += t[c2][q].y; acc.z += t[c2][q].z; acc.w += t[c2][q].w; }
-            v[4 * q] = __float_as_uint(acc.x); v[4 * q + 1] = __float_as_uint(acc.y);
-            v[4 * q + 2] = __float_as_uint(acc.z); v[4 * q + 3] = __float_as_uint(acc.w);
+            v[4 * q] = __float_as_uint(acc.x * rscale); v[4 * q + 1] = __float_as_uint(acc.y * rscale);
+            v[4 * q + 2] = __float_as_uint(acc.z * rscale); v[4 * q + 3] = __float_as_uint(acc.w * rscale);
           }
         }
       };

@@ -39,7 +39,7 @@ def test_workspace_bytes_and_config_validation(lib):
     big = binding.d2c_workspace_bytes(binding.make_config(inputs.LLADA_8B, 8, 4096))
     assert big > 2 * 32 * 8 * 4096 * 4096 * 2
     for field, val in [("head_dim", 96), ("d_model", 100), ("n_kv_heads", 3), ("max_seq", 10000), ("vocab", 1001),
-                       ("sigma", 0.0), ("flags", 16), ("stage2_candidates", 2)]:
+                       ("sigma", 0.0), ("flags", 32), ("stage2_candidates", 2)]:
         bad = binding.make_config(inputs.TOY, 1, 128)
         setattr(bad, field, val)
         assert binding.d2c_workspace_bytes(bad) == 0, field

@@ -52,10 +52,11 @@ WLS = {
 }
 
 
-@pytest.mark.parametrize("name", list(WLS))
-def test_prefill_then_partial_steps(name):
+@pytest.mark.parametrize("name,flags", [(n, 0) for n in WLS] + [("gqa_bias_3layers", 16), ("hd128_ragged_vocab", 16)])
+def test_prefill_then_partial_steps(name, flags):
+    """flags = 16: the same steps with the layers' RMSNorms folded into the GEMM epilogues around them."""
     wl = WLS[name]
-    pair = Pair(wl)
+    pair = Pair(wl, flags=flags)
     _prefill(pair)
     kc0 = pair.ctx.view("kcache").clone(); vc0 = pair.ctx.view("vcache").clone()
     for step, (k, p) in enumerate([(wl.k, wl.p), (wl.k, 0.1), (3, 0.5)]):
@@ -220,10 +221,11 @@ def test_truncated_rollout_depth():
 
 
 def test_kernel_variants_agree():
-    """The mma.sync GEMM / attention kernels and the one-SM tcgen05 GEMM give the same step within tolerance."""
+    """The mma.sync GEMM / attention kernels, the one-SM tcgen05 GEMM and the RMSNorms folded into the GEMM epilogues give the
+    same step within tolerance."""
     wl = inputs.Workload("hd128_big", inputs.TOY_HD128, 2, 300, 150, 60, "random", 8, 0.6, seed=9)
     ref = None
-    for flags in (0, 1 | 2, 4):                                       # default; portable GEMM + attention; one-SM GEMM
+    for flags in (0, 1 | 2, 4, 16):                                   # default; portable GEMM + attention; one-SM GEMM; RMSNorms folded into the GEMM epilogues
         pair = Pair(wl, flags=flags)
         pair.gpu_step(10 ** 6, 1.0)
         g = pair.gpu_step(wl.k, wl.p)
