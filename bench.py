@@ -238,7 +238,7 @@ def run_ours(args, rank, world, device):
     # dependent launches overlap as they do for a user.  Pass 2 repeats the step with one event at every phase
     # boundary (which serialises the launches) and gives the per-phase and per-kernel times; it runs long enough
     # (at least 100 steps of the short workloads) for the clock sampler to collect a usable number of readings.
-    prof_steps = args.steps if shape.n_layers > 4 else max(args.steps, 100)
+    prof_steps = args.profile_steps if args.profile_steps > 0 else (args.steps if shape.n_layers > 4 else max(args.steps, 100))
     sampler.start()
     per_step_ms, _ = timed_pass(False, args.steps)
     per_step_ms_profiled, phases = timed_pass(True, prof_steps)
@@ -507,6 +507,7 @@ def main():
     ap.add_argument("--rollout-layers", type=int, default=0,
                     help="roll the attention out over the first n layers only (the paper's Rollout-5 variant); 0 = all layers")
     ap.add_argument("--flags", type=int, default=0, help="D2C_FLAG_* bits for the context (kernel variants kept as cross-checks)")
+    ap.add_argument("--profile-steps", type=int, default=0, help="steps of the second, phase-timed pass (default: max(steps, 100) for the short workloads)")
     ap.add_argument("--no-extras", action="store_true", help="skip the labelled extra run at the paper's default p = 0.1")
     ap.add_argument("--scores", default="rollout", choices=["rollout", "zipf"],
                     help="stage-2 scores before each timed step: the prefill's rollout (default) or a seeded Zipf(1.0)")
