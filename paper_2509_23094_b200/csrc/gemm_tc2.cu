@@ -10,6 +10,15 @@
 // load); stage release and accumulator hand-over reach both CTAs through multicast tcgen05.commit.
 // Persistent: cluster c works on pair-tiles c, c + #clusters, ... with the row tile fastest.
 //
+// Ragged waves: when the tile count does not fill whole waves of clusters, tiles are not handed out one by one.
+// The clusters form groups of as many clusters as there are row tiles; the run of (column tile, pipeline stage)
+// pairs is cut into equal shares, one per group, and cluster j of a group walks its group's share for row tile j
+// (stream-K; the clusters of a group read the same weight k-blocks at about the same time, so the weights still
+// cross from HBM once).  A cluster whose share starts inside a tile parks that tile's partial sums (fp32) in its
+// own scratch slot first thing; the cluster holding the tile's first stages adds the parked parts in cluster
+// order and runs the epilogue.  Nobody waits for work that has not started, and an owner works on its shared
+// tile before its whole tiles, so the adding overlaps the next tile's MMAs.
+//
 // One thread issues every tcgen05.mma of a pair, and each step of its loop costs issue latency that does not
 // shrink with the tile: about 115 clocks for the full-barrier test, 58 per MMA and 95 for the commit (measured
 // with clock stamps on B200).  With one 64-wide k-block per pipeline stage that is ~560 clocks against the 512
@@ -71,6 +80,45 @@ __device__ __forceinline__ void mbar_arrive_even_cta(uint32_t bar) {
 
 struct Tc2Params { GemmArgs g; int* status; };
 
+// The pieces of work of one cluster, in order.  Round-robin: whole tiles (or (tile, part) items of a split-K
+// launch) cl, cl + #clusters, ...  Stream-K: the end of the tile its group's share starts in, then the start of
+// the tile the share ends in, then the whole tiles between.  All roles of both CTAs walk the same sequence.
+struct WorkIter {
+  int ncl, total, S, KT, KS;           // KS: pipeline stages per tile
+  int item;                            // round-robin: tile = item % total, part = item / total
+  int sk, MT, mt, phase;               // stream-K: on/off, row tiles, this cluster's row tile, next piece
+  int nt_tail, s_tail0, s_tail1;       // column tile and stages of the piece the share starts with (empty if s_tail1 <= s_tail0)
+  int nt_head, s_head1;                // column tile and end stage of the piece the share ends with (empty if 0)
+  int nt_full, n_full;                 // whole column tiles
+  __device__ void set_share(long long u0, long long u1) {
+    const int nt0 = (int)(u0 / KS), s0 = (int)(u0 - (long long)nt0 * KS);
+    nt_tail = nt0; s_tail0 = s_tail1 = 0;
+    if (s0 > 0) { s_tail0 = s0; s_tail1 = (int)min((long long)KS, s0 + (u1 - u0)); u0 += s_tail1 - s_tail0; }
+    nt_full = (int)(u0 / KS); n_full = (int)((u1 - u0) / KS);
+    nt_head = nt_full + n_full; s_head1 = (int)((u1 - u0) - (long long)n_full * KS);
+  }
+  __device__ bool next(int& tile, int& part, int& kb0, int& kb1) {
+    if (!sk) {
+      if (item >= total * S) return false;
+      tile = item % total; part = item / total;
+      kb0 = part * KT / S; kb1 = (part + 1) * KT / S;
+      item += ncl;
+      return true;
+    }
+    part = 0;
+    if (phase == 0) {
+      phase = 1;
+      if (s_tail1 > s_tail0) { tile = nt_tail * MT + mt; kb0 = s_tail0 * KSUB; kb1 = min(s_tail1 * KSUB, KT); return true; }
+    }
+    if (phase == 1) {
+      phase = 2;
+      if (s_head1 > 0) { tile = nt_head * MT + mt; kb0 = 0; kb1 = s_head1 * KSUB; return true; }
+    }
+    if (n_full > 0) { tile = nt_full * MT + mt; ++nt_full; --n_full; kb0 = 0; kb1 = KT; return true; }
+    return false;
+  }
+};
+
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -128,15 +176,27 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   // the issuing thread is the limit again).  Narrow tiles only pay when they fill the launch's waves of
   // clusters that much better; split-K (below) is preferred when few tiles are live.
   int bn = ACC_COLS;
+  const int KS = (KT + KSUB - 1) / KSUB;                     // pipeline stages per tile
+  // Stream-K (see the top of the file) when the evenly shared stages plus the hand-over (parking and adding a
+  // partial tile, about four stages' time) undercut whole waves of tiles.  Returns the number of groups.  Only the
+  // gate/up projection takes it: measured inside the step at 835 rows x d 4096 it gains 6 us of 143 there (and 6 %
+  // at 488 rows), while the QKV and down projections, whose shares hold at most two whole tiles to hide the adding
+  // behind, lose 3 and 8 us; the code below is written for every epilogue and was parity-tested with all of them.
+  auto stream_k_groups = [&](int col_tiles) {
+    if (EPI != EPI_SWIGLU || !sk_ok || MT <= 0 || 2 * MT > ncl || 2 * ncl > g.sk_max_tiles) return 0;
+    const int G = ncl / MT;
+    const long long stages = (long long)col_tiles * KS;
+    if (stages < 4LL * G) return 0;                          // every group gets a share worth starting
+    const long long shared = (stages + G - 1) / G + 4, in_waves = (long long)((MT * col_tiles + ncl - 1) / ncl) * KS;
+    return shared < in_waves ? G : 0;
+  };
   auto waves = [&](int out_cols) { const int t = MT * ((g.N + out_cols - 1) / out_cols); return (t + ncl - 1) / ncl; };
-  if (MT > 0 && (EPI == EPI_STORE || EPI == EPI_RESIDUAL)) {
-    const int t256 = MT * ((g.N + 255) / 256);
-    const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;
-    if (!will_split) {
-      float best = (float)waves(256);
-      if ((float)waves(128) * 0.75f < best) { best = (float)waves(128) * 0.75f; bn = 128; }
-      if ((float)waves(64) * 0.73f < best) { bn = 64; }
-    }
+  const int t256 = MT * ((g.N + 255) / 256);
+  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;
+  if (MT > 0 && (EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split && stream_k_groups((g.N + 255) / 256) == 0) {
+    float best = (float)waves(256);
+    if ((float)waves(128) * 0.75f < best) { best = (float)waves(128) * 0.75f; bn = 128; }
+    if ((float)waves(64) * 0.73f < best) { bn = 64; }
   }
   const int OUT_COLS = (EPI == EPI_SWIGLU) ? bn / 2 : bn;    // output columns per pair-tile
   const int NT = (g.N + OUT_COLS - 1) / OUT_COLS;
@@ -147,7 +207,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   int S = 1;
   if (sk_ok && total > 0 && total < ncl && 2 * total <= g.sk_max_tiles)
     S = max(1, min(min(ncl / total, KT / 8), 4));
-  const int items = total * S;
+  const int G = (S == 1 && bn == ACC_COLS) ? stream_k_groups(NT) : 0;
+  const long long sk_stages = (long long)NT * KS;            // stream-K: group q takes stages [q, q + 1) * sk_stages / G
+  WorkIter work;
+  work.ncl = ncl; work.total = max(total, 1); work.S = total > 0 ? S : 0; work.KT = KT; work.KS = KS; work.item = cl;
+  work.sk = G > 0; work.MT = max(MT, 1); work.mt = cl % max(MT, 1); work.phase = 0;
+  const int grp = cl / max(MT, 1);
+  if (G > 0) {
+    if (grp < G) work.set_share((long long)grp * sk_stages / G, (long long)(grp + 1) * sk_stages / G);
+    else work.set_share(0, 0);                               // clusters beyond the last whole group have no share
+  }
   const int b_box_rows = bn / 2;                             // weight rows this CTA brings in per k-block
 
   if (warp == 0) {
@@ -157,9 +226,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       bool ok = true;
       const uint32_t kb_bytes = 2 * (A_BYTES + (uint32_t)b_box_rows * TK * 2);   // both CTAs' boxes of one k-block
       const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
-      for (int item = cl; item < items && ok; item += ncl) {
-        const int tile = item % total, part = item / total;
-        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
+      WorkIter w = work;
+      int tile, part, k0, k1;
+      while (ok && w.next(tile, part, k0, k1)) {
         const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
         const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
         for (int kt = k0; kt < k1; kt += KSUB, ++it) {
@@ -193,9 +262,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((256u >> 4) << 24);
       const uint64_t desc0 = smem_desc_sw128(smem_base);     // A operand of stage 0, k-block 0
       int st = 0; uint32_t ph = 0;                           // ring position of the next stage
-      for (int item = cl; item < items && ok; item += ncl, ++tcount) {
-        const int part = item / total;
-        const int nk = (part + 1) * KT / S - part * KT / S;
+      WorkIter w = work;
+      int tile, part, k0, k1;
+      for (; ok && w.next(tile, part, k0, k1); ++tcount) {
+        const int nk = k1 - k0;
         const uint32_t buf = tcount & 1, use = tcount >> 1;
         if (!mbar_wait(acc_empty(buf), (use & 1) ^ 1, abortp, status, 34)) { ok = false; break; }
         const uint32_t tacc = tmem_acc + buf * ACC_COLS;
@@ -224,16 +294,18 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;
     uint32_t tcount = 0;
-    for (int item = cl; item < items; item += ncl, ++tcount) {
-      const int tile = item % total, part = item / total;
+    WorkIter w = work;
+    int tile, part, k0, k1;
+    for (; w.next(tile, part, k0, k1); ++tcount) {
       const uint32_t buf = tcount & 1, use = tcount >> 1;
       const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, nt = tile / MT, n0 = nt * OUT_COLS;
       const int row = m0 + lrow;
       const bool row_ok = row < n;
       const float rscale = folded_row_scale(g, row, row_ok);     // RMSNorm of the A rows folded into this GEMM (1 if none)
+      const bool sk_piece = S == 1 && (k0 > 0 || k1 < KT);       // part of a tile shared between clusters (stream-K)
       // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
       const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 33));
-      if (S > 1) {
+      if (S > 1 || sk_piece) {
         // ... and, where the four warps meet at named barriers below, for all of them together
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (*abortp) break;
@@ -243,10 +315,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       tc_fence_after();
       const uint32_t tbase = tmem_acc + buf * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       bool reduce = false;
+      int sk_parts = 0;                                          // parked parts this tile owner adds to its own
       const size_t slot_floats = (size_t)TM * ACC_COLS;
-      if (S > 1) {
+      const bool parks = S > 1 || (sk_piece && k0 > 0);          // this piece's sums go to scratch
+      if (parks) {
         const int acc_cols = bn;
-        float4* mine = reinterpret_cast<float4*>(g.sk_partials + ((size_t)(tile * S + part) * 2 + rank) * slot_floats);
+        const size_t slot = S > 1 ? (size_t)(tile * S + part) * 2 + rank : (size_t)cl * 2 + rank;
+        float4* mine = reinterpret_cast<float4*>(g.sk_partials + slot * slot_floats);
 #pragma unroll 1
         for (int c = 0; c < acc_cols / 32; ++c) {
           uint32_t v[32];
@@ -262,6 +337,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         tc_fence_before();
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (S == 1) {
+          // stream-K: tell the tile's owner (same row tile and CTA rank in the group holding the tile's first stage)
+          if (warp == 2 && lane == 0) {
+            for (int w4 = 0; w4 < 4; ++w4) mbar_arrive_even_cta(acc_empty(buf));
+            int og = grp - 1;
+            while (og > 0 && (long long)og * sk_stages / G > (long long)nt * KS) --og;
+            atomicAdd(&g.sk_counters[(og * MT + work.mt) * 2 + rank], 1);
+          }
+          continue;
+        }
         if (warp == 2 && lane == 0) {
           for (int w4 = 0; w4 < 4; ++w4) mbar_arrive_even_cta(acc_empty(buf));
           const int old = atomicAdd(&g.sk_counters[tile * 2 + rank], 1);
@@ -274,11 +359,41 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         asm volatile("bar.sync 1, 128;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
         if (!reduce) continue;
         __threadfence();
+      } else if (sk_piece) {
+        // stream-K tile owner: the groups after this one hold the rest of the tile's stages, up to the tile's end
+        for (int g2 = grp + 1; g2 < G && (long long)g2 * sk_stages / G < (long long)(nt + 1) * KS; ++g2) ++sk_parts;
+        if (warp == 2 && lane == 0) {
+          volatile int32_t* cnt = g.sk_counters + cl * 2 + rank;
+          const long long t0 = clock64();
+          bool there = true;
+          while (*cnt < sk_parts) {
+            if (*abortp || clock64() - t0 > kWaitCycles) { there = false; break; }
+            __nanosleep(64);
+          }
+          if (there) *cnt = 0;                                 // all parts are in: ready for the next launch
+          else if (!*abortp) { *abortp = 1; if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = 35; }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*abortp) break;
+        __threadfence();
       }
       auto load_chunk = [&](int col, uint32_t (&v)[32]) {     // 32 accumulator columns of this thread's row
         if (!reduce) {
           tmem_ld32(tbase + col, v);
           tmem_ld_wait();
+#pragma unroll 1
+          for (int j = 0; j < sk_parts; ++j) {                  // parked parts of this row tile, in group order
+            const float4* sp = reinterpret_cast<const float4*>(g.sk_partials + ((size_t)(cl + (1 + j) * MT) * 2 + rank) * slot_floats) +
+                               (size_t)(col >> 2) * TM + lrow;
+            float4 t[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) t[q] = row_ok ? __ldcg(sp + (size_t)q * TM) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              v[4 * q] = __float_as_uint(__uint_as_float(v[4 * q]) + t[q].x); v[4 * q + 1] = __float_as_uint(__uint_as_float(v[4 * q + 1]) + t[q].y);
+              v[4 * q + 2] = __float_as_uint(__uint_as_float(v[4 * q + 2]) + t[q].z); v[4 * q + 3] = __float_as_uint(__uint_as_float(v[4 * q + 3]) + t[q].w);
+            }
+          }
           if (g.in_ssq) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * rscale);
