@@ -8,7 +8,9 @@
 // k-block that is 32 KB of TMA traffic instead of 48 KB, which lifts the shared-memory bound of the
 // one-SM kernel.  TMA loads of both CTAs signal the even CTA's mbarrier (cta_group::2 form, no multicast
 // load); stage release and accumulator hand-over reach both CTAs through multicast tcgen05.commit.
-// Persistent: cluster c works on pair-tiles c, c + #clusters, ... with the row tile fastest.
+// Persistent: cluster c works on pair-tiles c, c + #clusters, ... with the row tile fastest.  Per CTA: warp 0
+// loads, warp 1 issues the MMAs, warps 2-9 run the epilogue, two per TMEM lane quarter, each on half of a
+// tile's columns (measured alone, the epilogue of the last tile of a launch is 3 us with one warp per quarter).
 //
 // Ragged waves: when the tile count does not fill whole waves of clusters, tiles are not handed out one by one.
 // The clusters form groups of as many clusters as there are row tiles; the run of (column tile, pipeline stage)
@@ -33,7 +35,8 @@ namespace d2c {
 namespace {
 
 constexpr int TM = 128, TK = 64;
-constexpr int TC_THREADS = 192;
+constexpr int EPI_WARPS = 8;                      // two per TMEM lane quarter: each takes half of a tile's columns
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int A_BYTES = TM * TK * 2;             // 16 KB: this CTA's rows
 constexpr int BH_BYTES = 128 * TK * 2;           // 16 KB: this CTA's half of the weight tile
 constexpr int SUB2 = A_BYTES + BH_BYTES;         // 32 KB per CTA and k-block
@@ -147,7 +150,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < ST2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }   // 4 epilogue warps x 2 CTAs
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 2 * EPI_WARPS); }   // epilogue warps of both CTAs
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -290,8 +293,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
-    const int quarter = warp & 3;
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int quarter = warp & 3;                             // TMEM lanes this warp may touch
+    const int ehalf = (warp - 2) >> 2;                        // which half of a tile's columns it takes
     const int lrow = quarter * 32 + lane;
     uint32_t tcount = 0;
     WorkIter w = work;
@@ -306,8 +310,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       // a wait that gave up ends the loop for the whole warp (the tcgen05.ld below is warp-collective) ...
       const bool got = __all_sync(0xffffffffu, mbar_wait(acc_full(buf), use & 1, abortp, status, 33));
       if (S > 1 || sk_piece) {
-        // ... and, where the four warps meet at named barriers below, for all of them together
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        // ... and, where the epilogue warps meet at named barriers below, for all of them together
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abortp) break;
       } else if (!got) {
         break;
@@ -323,7 +327,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const size_t slot = S > 1 ? (size_t)(tile * S + part) * 2 + rank : (size_t)cl * 2 + rank;
         float4* mine = reinterpret_cast<float4*>(g.sk_partials + slot * slot_floats);
 #pragma unroll 1
-        for (int c = 0; c < acc_cols / 32; ++c) {
+        for (int c = ehalf * (acc_cols / 64); c < (ehalf + 1) * (acc_cols / 64); ++c) {
           uint32_t v[32];
           tmem_ld32(tbase + c * 32, v);
           tmem_ld_wait();
@@ -336,11 +340,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         tc_fence_before();
         __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (S == 1) {
           // stream-K: tell the tile's owner (same row tile and CTA rank in the group holding the tile's first stage)
           if (warp == 2 && lane == 0) {
-            for (int w4 = 0; w4 < 4; ++w4) mbar_arrive_even_cta(acc_empty(buf));
+            for (int w4 = 0; w4 < EPI_WARPS; ++w4) mbar_arrive_even_cta(acc_empty(buf));
             int og = grp - 1;
             while (og > 0 && (long long)og * sk_stages / G > (long long)nt * KS) --og;
             atomicAdd(&g.sk_counters[(og * MT + work.mt) * 2 + rank], 1);
@@ -348,15 +352,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           continue;
         }
         if (warp == 2 && lane == 0) {
-          for (int w4 = 0; w4 < 4; ++w4) mbar_arrive_even_cta(acc_empty(buf));
+          for (int w4 = 0; w4 < EPI_WARPS; ++w4) mbar_arrive_even_cta(acc_empty(buf));
           const int old = atomicAdd(&g.sk_counters[tile * 2 + rank], 1);
           const int last = (old == S - 1) ? 1 : 0;
           if (last) g.sk_counters[tile * 2 + rank] = 0;      // every part has arrived: ready for the next launch
           sk_last = last;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         reduce = sk_last != 0;
-        asm volatile("bar.sync 1, 128;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
+        asm volatile("bar.sync 1, 256;" ::: "memory");      // sk_last may be rewritten only after everyone has read it
         if (!reduce) continue;
         __threadfence();
       } else if (sk_piece) {
@@ -373,7 +377,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (there) *cnt = 0;                                 // all parts are in: ready for the next launch
           else if (!*abortp) { *abortp = 1; if (atomicCAS(status, 0, D2C_ETIMEOUT) == 0) status[1] = 35; }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abortp) break;
         __threadfence();
       }
@@ -417,14 +421,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         }
       };
-      const EpiWarp ew{smem_base + (uint32_t)(ST2 * STAGE2) + (uint32_t)(quarter * kEpiStageBytes), m0 + quarter * 32, n, lane};
+      const EpiWarp ew{smem_base + (uint32_t)(ST2 * STAGE2) + (uint32_t)((warp - 2) * kEpiStageBytes), m0 + quarter * 32, n, lane};
       if (EPI == EPI_QKV_ROPE) {
-        epilogue_qkv_rope(load_chunk, g, ew, n0, OUT_COLS);
+        const int units = OUT_COLS >> 6;
+        epilogue_qkv_rope(load_chunk, g, ew, n0, OUT_COLS, ehalf * units / 2, (ehalf + 1) * units / 2);
       } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-        epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS);
+        const int units = OUT_COLS >> 5;
+        epilogue_rows<EPI>(load_chunk, g, ew, n0, OUT_COLS, ehalf * units / 2, (ehalf + 1) * units / 2);
       } else if (EPI == EPI_SWIGLU) {
-        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS);
-      } else {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
+        const int units = OUT_COLS >> 5;
+        epilogue_swiglu(load_chunk, g, ew, n0, OUT_COLS, ehalf * units / 2, (ehalf + 1) * units / 2);
+      } else if (ehalf == 0) {  // EPI_LMSTATS: one thread owns a whole row of the tile, so the statistics need no exchange
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {         // statistics are kept per 128 columns
           float mx = -INFINITY, sum = 0.f; int arg = 0x7fffffff;
@@ -483,7 +490,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
 template <int EPI>
 int launch_one(const GemmArgs& g, int* status, cudaStream_t st) {
-  const int smem = ST2 * STAGE2 + 1024 + 4 * kEpiStageBytes;   // stage ring, alignment slack, epilogue staging
+  const int smem = ST2 * STAGE2 + 1024 + EPI_WARPS * kEpiStageBytes;   // stage ring, alignment slack, epilogue staging
   static PerDevice attr_set;
   if (attr_set.first()) {
     D2C_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
