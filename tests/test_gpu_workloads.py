@@ -180,10 +180,12 @@ def test_llada_single_layer_1024_few_rows():
     assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
 
 
-@pytest.mark.parametrize("n_sel", [257, 323, 384, 385, 511, 835])
+@pytest.mark.parametrize("n_sel", [257, 323, 384, 385, 511, 600, 768, 835, 1023])
 def test_llada_single_layer_row_counts_around_the_pair_tile(n_sel):
-    """Selected-row counts with n mod 256 in {1, 67, 128, 129, 255}: the ragged last row tile of every projection
-    (fused QKV + rotary + cache scatter, residual, SwiGLU), all of its rows checked.  The rows are forced so
+    """Selected-row counts with n mod 256 in {0, 1, 67, 88, 128, 129, 255} over two, three and four row tiles: the
+    ragged last row tile of every projection (fused QKV + rotary + cache scatter, residual, SwiGLU), all of its rows
+    checked, and the gate/up projection's stream-K shares for every number of row tiles (tiles split between
+    clusters lie in every sampled row).  The rows are forced so
     that the count is exact; k = 0 and p = 0 select nothing else."""
     wl = inputs.WORKLOADS["llada1l_1024"]
     r = Runner(wl)
