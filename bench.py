@@ -275,6 +275,12 @@ def run_ours(args, rank, world, device):
     depth = args.rollout_layers if 0 < args.rollout_layers < shape.n_layers else shape.n_layers
     flops, byts = algorithmic_work(shape, B, L, n_b, n_m, depth)
     t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9))
+    # The same bound taken stage by stage: the LM head needs the last layer's output, so the layers (tensor-bound at
+    # many rows, weight-stream-bound at few) and the LM head (always bound by its weight stream) cannot overlap and
+    # their bounds add.  Reported beside the single max(), which lets the two resources overlap freely.
+    lm_flops, lm_byts = 2 * n_m * shape.d_model * shape.vocab, 2 * shape.d_model * shape.vocab
+    bound = lambda f, b: max(f / (peaks["bf16_tflops"] * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+    t_roof_serial = bound(flops - lm_flops, byts - lm_byts) + bound(lm_flops, lm_byts)
     # Denominator: the burst cuBLAS figure for a kernel inside a short step; the sustained one when the clock
     # record of the timed region shows the power cap holding the SM clock below 90 % of its maximum.
     capped = "sw_power_cap" in clocks.get("reasons", []) and clocks.get("sm_mhz", 0) < 0.9 * (clocks.get("sm_max_mhz") or 0)
@@ -311,6 +317,8 @@ def run_ours(args, rank, world, device):
                 "all_gemms": {"achieved": round(gemm_flops / (gemm_ms * 1e-3) / 1e12, 2) if gemm_ms > 0 else 0.0,
                               "ms_per_step": round(gemm_ms, 4)},
                 "step_roofline_ms": round(t_roof * 1e3, 4), "step_frac": round(t_roof * 1e3 / ms_per_step, 4),
+                "step_roofline_layers_then_lm_head_ms": round(t_roof_serial * 1e3, 4),
+                "step_frac_layers_then_lm_head": round(t_roof_serial * 1e3 / ms_per_step, 4),
                 "step_flops": flops, "step_bytes": byts}
     lm_ms = phases["lm_head"]["ms"] / prof_steps
     lm_bytes = 2 * d * shape.vocab
