@@ -195,9 +195,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   };
   auto waves = [&](int out_cols) { const int t = MT * ((g.N + out_cols - 1) / out_cols); return (t + ncl - 1) / ncl; };
   const int t256 = MT * ((g.N + 255) / 256);
-  const bool will_split = sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles;
-  if (MT > 0 && (EPI == EPI_STORE || EPI == EPI_RESIDUAL) && !will_split && stream_k_groups((g.N + 255) / 256) == 0) {
-    float best = (float)waves(256);
+  // Few tiles: either K is split (below), which costs a split tile about 28 k-blocks' time for parking, meeting and
+  // adding its parts, or the tiles are narrowed; with K = 4096 the narrow tiles win, with K = 12288 the split.
+  const int s256 = (sk_ok && 2 * t256 <= ncl && KT >= 16 && 2 * t256 <= g.sk_max_tiles) ? max(1, min(min(ncl / max(t256, 1), KT / 8), 4)) : 1;
+  if (MT > 0 && (EPI == EPI_STORE || EPI == EPI_RESIDUAL) && stream_k_groups((g.N + 255) / 256) == 0) {
+    float best = s256 > 1 ? ((float)((KT + s256 - 1) / s256) + 28.f) / (float)KT : (float)waves(256);
     if ((float)waves(128) * 0.75f < best) { best = (float)waves(128) * 0.75f; bn = 128; }
     if ((float)waves(64) * 0.73f < best) { bn = 64; }
   }
