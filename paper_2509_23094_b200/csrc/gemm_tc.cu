@@ -91,8 +91,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
   const uint32_t tmem_acc = tmem_slot;
   volatile int* abortp = &abort_flag;
 
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
+  // The live row count is read, and the weight boxes of the first ring fill are requested, before the wait on the
+  // preceding kernel: neither is that kernel's output (the count is the selection kernel's, which has completed
+  // before any GEMM's CTA runs: every kernel between it and a GEMM waits for its own predecessor before it lets
+  // its successor launch, or is a GEMM behind such a kernel).  What the predecessor may have written (A rows, the
+  // residual, split-K scratch) is touched only behind each role's own griddepcontrol.wait.
   const int n = max(*g.n_rows, 0);
   const int MT = (n + TM - 1) / TM;
   const int KT = g.K / TK, G = gridDim.x;
@@ -147,31 +150,52 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     if (lane == 0) {
       uint32_t it = 0;                                        // stages issued so far (ring position)
       bool ok = true;
+      auto load_w = [&](uint32_t sb, int kc, int n0, uint32_t bar) {      // the weight rows of one k-block
+        if (bn == 64) {
+          tma_load_2d(sb, &tmB64, kc, n0, bar);
+        } else {
+          tma_load_2d(sb, &tmB, kc, n0, bar);
+          if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kc, n0, bar);
+          else if (bn == 256) tma_load_2d(sb + 128 * TK * 2, &tmB, kc, n0 + 128, bar);
+        }
+      };
+      auto a_box_rows = [&](int m0) { const int rows = n - m0; return rows <= 32 ? 32 : (rows <= 64 ? 64 : 128); };   // live rows of a tile: load no more than needed
+      uint32_t early = 0;                                     // stages whose byte count and weight boxes are already out
+      for (int item = blockIdx.x; item < items && early < (uint32_t)nst; item += G) {
+        const int tile = item % total, part = item / total;
+        const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
+        const int m0 = (tile % MT) * TM, n0 = (tile / MT) * OUT_COLS;
+        const uint32_t kb_bytes = (uint32_t)a_box_rows(m0) * TK * 2 + (uint32_t)b_rows * TK * 2;
+        for (int kt = k0; kt < k1 && early < (uint32_t)nst; kt += ksub, ++early) {
+          const int nsub = min(ksub, k1 - kt);
+          mbar_expect_tx(full_bar(early), (uint32_t)nsub * kb_bytes);
+#pragma unroll
+          for (int u = 0; u < KSUB; ++u)
+            if (u < nsub) load_w(smem_base + early * stage_bytes + u * sub_bytes + a_rows_max * TK * 2, (kt + u) * TK, n0, full_bar(early));
+        }
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (g.clock_probe && blockIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
       for (int item = blockIdx.x; item < items && ok; item += G) {
         const int tile = item % total, part = item / total;
         const int k0 = part * KT / S, k1 = (part + 1) * KT / S;
         const int m0 = (tile % MT) * TM, n0 = (tile / MT) * OUT_COLS;
-        const int rows = n - m0;                              // live rows of this tile: load no more than needed
-        const CUtensorMap* ma = rows <= 32 ? &tmA32 : (rows <= 64 ? &tmA64 : &tmA128);
-        const uint32_t kb_bytes = (rows <= 32 ? 32 : (rows <= 64 ? 64 : 128)) * TK * 2 + (uint32_t)b_rows * TK * 2;
+        const int arows = a_box_rows(m0);
+        const CUtensorMap* ma = arows == 32 ? &tmA32 : (arows == 64 ? &tmA64 : &tmA128);
+        const uint32_t kb_bytes = (uint32_t)arows * TK * 2 + (uint32_t)b_rows * TK * 2;
         for (int kt = k0; kt < k1; kt += ksub, ++it) {
           const int s = it % nst;
           const int nsub = min(ksub, k1 - kt);
+          const bool fresh = it >= early;                     // not one of the stages started before the wait
           if (!mbar_wait(empty_bar(s), ((it / nst) & 1) ^ 1, abortp, status, 1)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
+          if (fresh) mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
 #pragma unroll
           for (int u = 0; u < KSUB; ++u) {
             if (u < nsub) {
               const uint32_t sa = smem_base + s * stage_bytes + u * sub_bytes, sb = sa + a_rows_max * TK * 2;
               const int kc = (kt + u) * TK;
               tma_load_2d(sa, ma, kc, m0, full_bar(s));
-              if (bn == 64) {
-                tma_load_2d(sb, &tmB64, kc, n0, full_bar(s));
-              } else {
-                tma_load_2d(sb, &tmB, kc, n0, full_bar(s));
-                if (EPI == EPI_SWIGLU) tma_load_2d(sb + 128 * TK * 2, &tmB2, kc, n0, full_bar(s));
-                else if (bn == 256) tma_load_2d(sb + 128 * TK * 2, &tmB, kc, n0 + 128, full_bar(s));
-              }
+              if (fresh) load_w(sb, kc, n0, full_bar(s));
             }
           }
         }
@@ -224,6 +248,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA128, const __grid_constant
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;                             // TMEM lanes this warp may touch
     const int lrow = quarter * 32 + lane;
+    asm volatile("griddepcontrol.wait;" ::: "memory");        // the residual, the scratch and the outputs belong to the step's chain
     uint32_t tcount = 0;
     for (int item = blockIdx.x; item < items; item += G, ++tcount) {
       const int tile = item % total, part = item / total;

@@ -167,8 +167,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const uint32_t tmem_acc = tmem_slot;
   volatile int* abortp = &abort_flag;
 
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (g.clock_probe && blockIdx.x == 0 && threadIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
+  // The live row count is read, and the weight boxes of the first ring fill are requested, before the wait on the
+  // preceding kernel: neither is that kernel's output.  The count was written by the selection kernel at the start
+  // of the step, and every kernel between it and a GEMM either waits for its own predecessor before it lets its
+  // successor launch (the row kernels, attention) or is a GEMM behind such a kernel, so selection has completed
+  // before any GEMM's CTA runs.  Everything the predecessor may have written (A rows, the residual, split-K
+  // scratch) is touched only behind each role's own griddepcontrol.wait.
   const int n = *g.n_rows;
   const int MT = (max(n, 0) + 2 * TM - 1) / (2 * TM);
   const int KT = g.K / TK;
@@ -231,22 +235,40 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       bool ok = true;
       const uint32_t kb_bytes = 2 * (A_BYTES + (uint32_t)b_box_rows * TK * 2);   // both CTAs' boxes of one k-block
       const CUtensorMap* mb = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : (bn == 256 ? &tmB : (bn == 128 ? &tmB64 : &tmB32));
-      WorkIter w = work;
       int tile, part, k0, k1;
+      uint32_t early = 0;                                     // stages whose byte count and weight boxes are already out
+      {
+        WorkIter w = work;
+        while (early < (uint32_t)ST2 && w.next(tile, part, k0, k1)) {
+          const int n0 = (tile / MT) * OUT_COLS;
+          const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
+          for (int kt = k0; kt < k1 && early < (uint32_t)ST2; kt += KSUB, ++early) {
+            const int nsub = min(KSUB, k1 - kt);
+            if (leader) mbar_expect_tx(full_bar(early), (uint32_t)nsub * kb_bytes);
+#pragma unroll
+            for (int u = 0; u < KSUB; ++u)
+              if (u < nsub) tma_load_2d_pair(smem_base + early * STAGE2 + u * SUB2 + A_BYTES, mb, (kt + u) * TK, brow, full_bar(early));
+          }
+        }
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (g.clock_probe && blockIdx.x == 0) { g.clock_probe[0] = clock64(); g.clock_probe[1] = global_timer_ns(); }
+      WorkIter w = work;
       while (ok && w.next(tile, part, k0, k1)) {
         const int m0 = (tile % MT) * 2 * TM + (int)rank * TM, n0 = (tile / MT) * OUT_COLS;
         const int brow = (EPI == EPI_SWIGLU) ? n0 : n0 + (int)rank * (bn / 2);
         for (int kt = k0; kt < k1; kt += KSUB, ++it) {
           const int s = it % ST2;
           const int nsub = min(KSUB, k1 - kt);
+          const bool fresh = it >= early;                     // not one of the stages started before the wait
           if (!mbar_wait(empty_bar(s), ((it / ST2) & 1) ^ 1, abortp, status, 31)) { ok = false; break; }
-          if (leader) mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
+          if (leader && fresh) mbar_expect_tx(full_bar(s), (uint32_t)nsub * kb_bytes);
 #pragma unroll
           for (int u = 0; u < KSUB; ++u) {
             if (u < nsub) {
               const uint32_t sa = smem_base + s * STAGE2 + u * SUB2, sb = sa + A_BYTES;
               tma_load_2d_pair(sa, &tmA, (kt + u) * TK, m0, full_bar(s));
-              tma_load_2d_pair(sb, mb, (kt + u) * TK, brow, full_bar(s));
+              if (fresh) tma_load_2d_pair(sb, mb, (kt + u) * TK, brow, full_bar(s));
             }
           }
         }
@@ -298,6 +320,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int quarter = warp & 3;                             // TMEM lanes this warp may touch
     const int ehalf = (warp - 2) >> 2;                        // which half of a tile's columns it takes
+    asm volatile("griddepcontrol.wait;" ::: "memory");        // the residual, the scratch and the outputs belong to the step's chain
     const int lrow = quarter * 32 + lane;
     uint32_t tcount = 0;
     WorkIter w = work;
