@@ -29,8 +29,13 @@ void count_launch(int n);
     }                                                                                  \
   } while (0)
 // Programmatic dependent launch: every kernel of the step is launched with the stream-serialisation
-// attribute and starts with pdl_prologue(), which waits for the preceding kernel's results and then
-// lets the following kernel begin its own launch, so launch latency overlaps the predecessor's tail.
+// attribute.  All but the GEMMs start with pdl_prologue(), which waits for the preceding kernel's results and
+// then lets the following kernel begin its own launch, so launch latency overlaps the predecessor's tail.  The
+// tcgen05 GEMMs let their successor launch first, set up barriers and TMEM, read the row count and request their
+// first weight boxes, and wait only before they touch what the predecessor wrote.  That is sound because a
+// pdl_prologue() kernel stands between the selection kernel, which writes the counts, and every GEMM: nothing
+// behind that kernel can run before selection has completed.  (The same order in the attention kernels, whose
+// loads all depend on the predecessor, measured no different and is not used.)
 #ifdef __CUDACC__
 __device__ __forceinline__ long long global_timer_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 __device__ __forceinline__ void pdl_prologue() {
