@@ -136,6 +136,7 @@ struct d2c_ctx {
   long long hint_step[2] = {-1, -1};     // step number whose count the word holds
   long long step_no = 0;
   bool few_rows = false;                 // this step's regime: at most 128 rows expected
+  bool one_sm_gemm = false;              // at most 384 rows expected: the projections run on the one-SM kernel
   int used_batch = 0, used_seq = 0;      // the (batch, seq_len) of the first step: the per-position state is laid out for it
   // d2c_step_host: the device-to-host copy of the hidden rows runs on its own stream, ordered after the
   // last layer by an event, so that it overlaps the LM head and the rollout
@@ -204,8 +205,11 @@ static int gemm(d2c_ctx* ctx, const GemmArgs& g, GemmEpilogue epi) {
   if (ctx->cfg.flags & D2C_FLAG_PORTABLE_GEMM) return launch_gemm_mma(g, epi, ctx->run);
   // The LM head runs on few rows and is bound by the weight stream: the one-SM kernel sizes its A boxes to the
   // live rows, a pair would load a second, empty row tile.
-  const bool few_rows = ctx->few_rows;                      // weight-streaming regime
-  if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && !few_rows && gemm_tc2_supported(g))
+  // Up to three 128-row tiles the one-SM kernel wins: its row tiles pad 257..384 rows to 384 where a pair tile pads
+  // them to 512, and below 129 rows it streams weights with K split over the SMs.  Measured on one layer at
+  // L = 1024 (step, ms): 204 rows 0.418 -> 0.398, 292 rows 0.456 -> 0.423, 381 rows 0.460 -> 0.427; from 470 rows
+  // on the pairs win (0.461 against 0.481; 561 rows 0.529 against 0.540).
+  if (!(ctx->cfg.flags & D2C_FLAG_ONE_SM_GEMM) && epi != EPI_LMSTATS && !ctx->one_sm_gemm && gemm_tc2_supported(g))
   {
     GemmArgs g2 = g;
     g2.sk_partials = ctx->buf.sk_partials; g2.sk_counters = ctx->buf.sk_counters; g2.sk_max_tiles = kSkMaxTiles;
@@ -388,6 +392,7 @@ int d2c_step(d2c_ctx* ctx, const d2c_step_args* a, const d2c_step_out* out) {
     expect_rows = *reinterpret_cast<volatile int32_t*>(ctx->hint_host[prev]);
   }
   ctx->few_rows = expect_rows <= 128;
+  ctx->one_sm_gemm = expect_rows <= 384;
   const bool few_rows = ctx->few_rows;
   const bool abar_aside = overlap && (c.n_layers == 1 || few_rows);
   bool abar_pending = false, rollout_done = false;

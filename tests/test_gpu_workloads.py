@@ -206,10 +206,11 @@ def test_llada_single_layer_row_counts_around_the_pair_tile(n_sel):
     assert torch.equal(kc1[:, 0, :L][:, keep], kc0[:, 0, :L][:, keep]) and torch.equal(vc1[:, 0, :L][:, keep], vc0[:, 0, :L][:, keep])
 
 
-@pytest.mark.parametrize("n_sel", [1, 33, 64, 100, 128])
+@pytest.mark.parametrize("n_sel", [1, 33, 64, 100, 128, 129, 200, 257, 384])
 def test_llada_single_layer_few_forced_rows(n_sel):
-    """At most 128 rows: from the second such step on the projections run on the one-SM kernel, every tile's K
-    range split over several SMs whose parts each finish a share of the tile's columns."""
+    """At most 384 rows: from the second such step on the projections run on the one-SM kernel (one to three
+    128-row tiles), every tile's K range split over several SMs whose parts each finish a share of the tile's
+    columns; up to 128 rows the probabilities pass also moves beside the main stream."""
     wl = inputs.WORKLOADS["llada1l_1024"]
     r = Runner(wl)
     B, L = wl.batch, wl.seq_len
