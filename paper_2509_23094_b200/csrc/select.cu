@@ -60,7 +60,10 @@ __device__ __forceinline__ float clean_score(float x) { return (x > 0.f && x < I
 
 // Shared scratch of the threshold search.
 struct RadixScratch {
-  unsigned long long hist[256];            // per digit: the weight sum of the members that carry it
+  // per digit: the weight sum of the members that carry it, kept as three 32-bit sums of 17-bit pieces of the
+  // weights (weights stay below 2^51, 8192 positions x 2^17 below 2^32): 32-bit shared-memory atomics are native,
+  // the 64-bit ones took about seven clocks per lane whatever the address (6700 of a 1024-position pass's clocks)
+  uint32_t hist[3][256];
   unsigned long long warp_buf[32];
   unsigned long long total;
   unsigned long long above;
@@ -104,11 +107,15 @@ __device__ __forceinline__ void take_until_crossed(const uint32_t* vb, int L, Me
         unsigned long long w = m ? weight(vb[j]) : 0ull;
         const int leader = __ffs(act) - 1;
         const uint32_t d0 = __shfl_sync(0xffffffffu, d, leader);
-        if (__all_sync(0xffffffffu, !m || d == d0)) {
+        const bool one_digit = __all_sync(0xffffffffu, !m || d == d0);
+        if (one_digit)
           for (int o = 16; o > 0; o >>= 1) w += shfl_xor_u64(w, o);
-          if (lane == leader && w) atomicAdd(&rs.hist[d0], w);
-        } else if (m && w) {
-          atomicAdd(&rs.hist[d], w);
+        if (one_digit ? lane == leader : m) {
+          // (a warp's sum of 32 weights may carry into bit 51 and above: the top piece takes all the high bits)
+          const uint32_t w0 = (uint32_t)(w & 0x1FFFFull), w1 = (uint32_t)((w >> 17) & 0x1FFFFull), w2 = (uint32_t)(w >> 34);
+          if (w0) atomicAdd(&rs.hist[0][d], w0);
+          if (w1) atomicAdd(&rs.hist[1][d], w1);
+          if (w2) atomicAdd(&rs.hist[2][d], w2);
         }
       }
     }
@@ -119,8 +126,8 @@ __device__ __forceinline__ void take_until_crossed(const uint32_t* vb, int L, Me
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int bin = 255 - (8 * lane + k);
-        w[k] = rs.hist[bin];
-        rs.hist[bin] = 0;
+        w[k] = (unsigned long long)rs.hist[0][bin] + ((unsigned long long)rs.hist[1][bin] << 17) + ((unsigned long long)rs.hist[2][bin] << 34);
+        rs.hist[0][bin] = 0; rs.hist[1][bin] = 0; rs.hist[2][bin] = 0;
         sum += w[k];
       }
       unsigned long long inc = sum;
@@ -204,7 +211,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
     cb[i] = __float_as_uint(clean_score(cs[i]));
   }
   for (int r = tid; r < min(a.phi_len, kPhiMax); r += kSelThreads) s_phi[r] = a.phi_q30[r];
-  for (int i = tid; i < 256; i += kSelThreads) rsc.hist[i] = 0;
+  for (int i = tid; i < 3 * 256; i += kSelThreads) (&rsc.hist[0][0])[i] = 0;
   if (tid == 0) { s_nm = 0; s_mass = 0; s_lo = 0xFFFFFFFFu; s_hi = 0u; }
   __syncthreads();
 
@@ -284,12 +291,20 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
       for (int i = tid; i < L; i += kSelThreads)
         if (in1[i]) flags[i] = F_SEL | F_MSTAR;
     } else if (take > 0 && nm <= kRankMax) {
-      // rank of a listed position = how many others come before it; every thread reads the same entry at a time
-      for (int e = tid; e < nm; e += kSelThreads) {
-        const unsigned long long mine = mlist[e];
+      // rank of a listed position = how many others come before it; a group of tpe lanes (a power of two, inside
+      // one warp) shares a position and each counts every tpe-th entry
+      int tpe = 1;
+      while (tpe < 32 && 2 * tpe * nm <= kSelThreads) tpe <<= 1;
+      const int sub = tid & (tpe - 1), groups = kSelThreads / tpe;
+      for (int e0 = 0; e0 < nm; e0 += groups) {
+        const int e = e0 + tid / tpe;
+        const bool live = e < nm;
+        const unsigned long long mine = live ? mlist[e] : 0ull;
         int rank = 0;
-        for (int f = 0; f < nm; ++f) rank += mlist[f] > mine ? 1 : 0;
-        if (rank < take) flags[0xFFFFFFFFu - (uint32_t)(mine & 0xFFFFFFFFull)] = F_SEL | F_MSTAR;
+        if (live)
+          for (int f = sub; f < nm; f += tpe) rank += mlist[f] > mine ? 1 : 0;
+        for (int o = 1; o < tpe; o <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+        if (live && sub == 0 && rank < take) flags[0xFFFFFFFFu - (uint32_t)(mine & 0xFFFFFFFFull)] = F_SEL | F_MSTAR;
       }
     } else if (take > 0) {
       const unsigned long long want = (unsigned long long)take;
@@ -315,8 +330,27 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
       atomicMin(&s_lo, lo); atomicMax(&s_hi, hi);
     }
     __syncthreads();
-    const double thr = __dmul_rn((double)a.p, __ull2double_rn(s_mass));
-    take_until_crossed(cb, L, cand, mass, [&](unsigned long long w) { return __ull2double_rn(w) > thr; }, flags, (uint8_t)F_SEL, rsc,
+    // (p above 1 selects every candidate, as p = 1 does: the total never exceeds itself)
+    const double thr = __dmul_rn(fmin((double)a.p, 1.0), __ull2double_rn(s_mass));
+    // The prefix's mass has crossed when double(mass) > thr.  double() is monotone, so that is mass >= T for the
+    // smallest integer T whose double exceeds thr, and the search compares integers.  Below 2^52 every integer is
+    // its own double: T = floor(thr) + 1; above, T lies within 2048 of floor(thr) (doubles are at most 1024 apart
+    // below 2^63) and a bisection finds it.
+    unsigned long long T;
+    {
+      const unsigned long long fl = __double2ull_rd(thr);
+      if (thr < 4503599627370496.0) {
+        T = fl + 1ull;
+      } else {
+        unsigned long long lo_t = fl - 2048ull, hi_t = fl + 2049ull;        // double(lo_t) <= thr < double(hi_t)
+        while (hi_t - lo_t > 1ull) {
+          const unsigned long long mid = lo_t + ((hi_t - lo_t) >> 1);
+          if (__ull2double_rn(mid) > thr) hi_t = mid; else lo_t = mid;
+        }
+        T = hi_t;
+      }
+    }
+    take_until_crossed(cb, L, cand, mass, [&](unsigned long long w) { return w >= T; }, flags, (uint8_t)F_SEL, rsc,
                        s_lo, max(s_hi, s_lo));
   }
 
