@@ -255,7 +255,8 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       for (int j = 0; j < T && ok; ++j) {
         const int sp = dbuf ? (j & 1) : q;                          // S/P buffer of this tile
         const uint32_t ts = tm + sp * 256 + lane_base;
-        if (!mbar_wait(B(7 + sp), (dbuf ? (j >> 1) : j) & 1, abortp, status, 18)) { ok = false; break; }
+        // a wait that gave up ends the loop for the whole warp: the tcgen05.ld / st below are warp-collective
+        if (!__all_sync(0xffffffffu, mbar_wait(B(7 + sp), (dbuf ? (j >> 1) : j) & 1, abortp, status, 18))) { ok = false; break; }
         tc_fence_after();
         const int key0 = j * AKEYS;
         const bool full = key0 + AKEYS <= L;
@@ -263,23 +264,19 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(ts + c * 32, sv[c]);
         tmem_ld_wait();
+        if (!full) {                                                // last, ragged key tile: keys past L score -inf (probability 0)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (key0 + c * 32 + i >= L) sv[c][i] = __float_as_uint(-INFINITY);
+        }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        if (full) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2)                             // three-input maximum: two scores per instruction
-              mx4[(i >> 1) & 3] = fmax3(mx4[(i >> 1) & 3], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float f = __uint_as_float(sv[c][i]);
-              if (key0 + c * 32 + i < L) mx4[i & 3] = fmaxf(mx4[i & 3], f);
-            }
-          }
+          for (int i = 0; i < 32; i += 2)                               // three-input maximum: two scores per instruction
+            mx4[(i >> 1) & 3] = fmax3(mx4[(i >> 1) & 3], __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
         }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
         const bool raise = mx > m_used + kRescaleStep;              // always true on the first tile
@@ -288,7 +285,7 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           if (raise) m_used = mx;
           l *= alpha;
           if (j > 0) {                                              // O holds the sum of tiles 0..j-1: rescale it in place
-            if (!mbar_wait(B(11 + q), (j - 1) & 1, abortp, status, 17)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(B(11 + q), (j - 1) & 1, abortp, status, 17))) { ok = false; break; }
             tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
@@ -313,12 +310,7 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           for (int i = 0; i < 16; ++i) {
             float x0, x1;
             unpack2(fma2(pack2(__uint_as_float(sv[c][2 * i]), __uint_as_float(sv[c][2 * i + 1])), sc2, nm2), x0, x1);
-            float p0 = exp2f(x0), p1 = exp2f(x1);
-            if (!full) {
-              const int k = key0 + c * 32 + 2 * i;
-              if (k >= L) p0 = 0.f;
-              if (k + 1 >= L) p1 = 0.f;
-            }
+            const float p0 = exp2f(x0), p1 = exp2f(x1);
             rs2[i & 3] = add2(rs2[i & 3], pack2(p0, p1));
             pk[i] = pack_bf16(p0, p1);
           }
@@ -334,7 +326,7 @@ attn_fwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         __syncwarp();
         if (lane == 0) mbar_arrive(B(9 + sp));
       }
-      if (ok) ok = mbar_wait(B(11 + q), (T - 1) & 1, abortp, status, 19);
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(B(11 + q), (T - 1) & 1, abortp, status, 19));
       tc_fence_after();
       if (ok) {
         const bool row_ok = lrow < nrows;
@@ -473,7 +465,7 @@ attn_abar_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     for (int h = 0; h < nh && ok; ++h) {
       const int sb = h & 1;
       const float e = row_ok ? a.lse[(size_t)(r0 + lrow) * a.hq + h_first + h] * kLog2e : 0.f;
-      if (!mbar_wait(SF(sb), (h >> 1) & 1, abortp, status, 26)) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(SF(sb), (h >> 1) & 1, abortp, status, 26))) { ok = false; break; }   // whole warp or nobody: tcgen05.ld below
       tc_fence_after();
       uint32_t v[2][32];
       tmem_ld32(tm + sb * 128 + lane_base + half * 64, v[0]);
